@@ -1,0 +1,186 @@
+/*
+ * codistill.h -- C ABI of the fused codistillation objective (loss forward + gradient
+ * with respect to the logits) for NVIDIA B200 (sm_100a).
+ *
+ * The operation is the per-model objective inside the update of Algorithm 1
+ * ("Codistillation") of "A Closer Look at Codistillation for Distributed Training"
+ * (arXiv 2010.02838): for model i with logits z and peers z^(j), j != i,
+ *
+ *     loss_row = L(y, z) + alpha * 1/(n-1) * sum_{j != i} D(z, z^(j))
+ *
+ * where L is the cross-entropy of softmax(z) against the label y (Section 2: "a standard
+ * supervised loss function L (e.g., cross-entropy ...)") and D is, as in the paper's
+ * experiments (Appendix, "Implementation Details"), the mean squared error between the raw,
+ * un-centred logits of the two models.  The KL divergence between temperature softmaxes
+ * that Section 2 attributes to earlier work is available as a second form of D.  The
+ * gradient is taken with respect to model i's logits only; the peers are constants
+ * (Algorithm 1 differentiates with respect to theta_i alone; Section 3).
+ *
+ * Conventions common to every entry point
+ *   - Unless a parameter says HOST, a pointer is a DEVICE pointer owned by the caller; the
+ *     library never frees or keeps it.  Inputs are never written.  grad_logits must not
+ *     alias an input.
+ *   - Work is enqueued on the caller's stream and the call returns immediately; outputs are
+ *     valid once that stream has been synchronised.
+ *   - Return value: CODISTILL_OK, or a CODISTILL_ERR_* code for anything the host can
+ *     check, in which case nothing was launched.  Conditions only the device can see set
+ *     bits in *dev_status (CODISTILL_DEV_*).  Nothing traps, aborts or prints.
+ *   - Tensors are row-major [rows, classes] with a common row pitch `row_stride` (in
+ *     elements, >= classes) for logits, every peer and grad_logits.
+ *   - rows == 0 is valid: reduced loss 0, counters 0.
+ *   - NaN / Inf inputs propagate by IEEE rules and are outside the tested domain.
+ */
+#ifndef CODISTILL_H_
+#define CODISTILL_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+/* host-side return codes */
+enum {
+  CODISTILL_OK = 0,
+  CODISTILL_ERR_NULL = 1,        /* a required pointer is NULL */
+  CODISTILL_ERR_SHAPE = 2,       /* n < 1, rows < 0, classes < 1, row_stride < classes, sizes too large */
+  CODISTILL_ERR_DTYPE = 3,       /* dtype is not CODISTILL_F32 / CODISTILL_BF16 */
+  CODISTILL_ERR_PARAM = 4,       /* temperature <= 0, non-finite alpha, label_smoothing outside [0,1), bad enum */
+  CODISTILL_ERR_UNSUPPORTED = 5, /* valid request this build cannot serve (e.g. n - 1 > CODISTILL_MAX_PEERS) */
+  CODISTILL_ERR_CUDA = 6,        /* a CUDA runtime call failed; the CUDA error is left for cudaGetLastError */
+  CODISTILL_ERR_WORKSPACE = 7    /* workspace NULL, misaligned (256 B) or smaller than codistill_workspace_bytes */
+};
+
+/* element type of logits, peers and grad_logits */
+enum { CODISTILL_F32 = 0, CODISTILL_BF16 = 1 };
+
+/* form of the distillation distance D */
+enum {
+  CODISTILL_DIST_MSE_LOGITS = 0, /* D(z, z') = 1/C * sum_c (z_c - z'_c)^2 (Appendix "Implementation Details") */
+  CODISTILL_DIST_KL_SOFTMAX = 1  /* D(z, z') = T^2 * KL(softmax(z'/T) || softmax(z/T)) (Section 2, earlier work) */
+};
+
+/* how the n-1 peers enter D */
+enum {
+  CODISTILL_PEERS_PAIRWISE_MEAN = 0, /* 1/(n-1) * sum_j D(z, z^(j))      -- Algorithm 1 as printed          */
+  CODISTILL_PEERS_MEAN_TARGET = 1    /* D(z, zbar), zbar = 1/(n-1) * sum_j z^(j) -- distance to the averaged peer */
+};
+
+/* reduction over rows; the gradient is the gradient of the reduced loss */
+enum { CODISTILL_REDUCE_MEAN_VALID = 0, CODISTILL_REDUCE_SUM = 1 };
+
+/* bits OR-ed into *dev_status by the kernels */
+enum {
+  CODISTILL_DEV_BAD_LABEL = 1, /* a valid row had a label outside [0, classes); that row was treated as masked */
+  CODISTILL_DEV_TIMEOUT = 2,   /* a bounded wait on an asynchronous copy expired; outputs are not to be trusted */
+  CODISTILL_DEV_ASSERT = 4     /* an internal consistency check failed */
+};
+
+#define CODISTILL_MAX_PEERS 31 /* n <= 32 */
+
+/* layout of counters[]: [0] n_valid, [1] n_masked, [2] n_correct, [3 + j] n_agree with peer j */
+#define CODISTILL_COUNTERS_FIXED 3
+
+/*
+ * Full parameter block (Algorithm 1's objective with every knob this library exposes).
+ *
+ *   struct_bytes     sizeof(codistill_params_t) as seen by the caller (ABI check).
+ *   logits           [rows, row_stride] own logits z of model i.
+ *   peer_logits      HOST array of n-1 device pointers, each [rows, row_stride]; may be NULL when n == 1.
+ *   labels           [rows] int32 class ids y.
+ *   mask             [rows] uint8, non-zero = valid row; NULL = all rows valid.  The paper does not
+ *                    mention padding; masked rows get zero loss and an all-zero gradient row.
+ *   n                number of codistilled models (n == 1: plain training, no distillation term).
+ *   alpha            penalty coefficient alpha^k of Algorithm 1.  alpha == 0 skips the term.
+ *   temperature      T > 0; used by the KL form only (the paper's MSE form has no temperature).
+ *   label_smoothing  eps in [0,1): target q = (1-eps)*onehot(y) + eps/C for the task loss.
+ *   row_loss         [rows] float output, per-row loss (0 for masked rows); may be NULL.
+ *   reduced_loss     [1] float output: sum over valid rows (SUM) or that / max(n_valid,1) (MEAN_VALID).
+ *   grad_logits      [rows, row_stride] output in `dtype` (bf16: round-to-nearest-even); NULL = forward only.
+ *                    Only the first `classes` elements of each row are written.
+ *   counters         [3 + (n-1)] int64 output (bit-exact integers), may be NULL:
+ *                    n_valid, n_masked, n_correct = #{valid r: argmax z = y},
+ *                    n_agree[j] = #{valid r: argmax z = argmax z^(j)}; lowest index wins ties.
+ *   dev_status       [1] int32 output, CODISTILL_DEV_* bits; may be NULL.
+ *   workspace        scratch of at least codistill_workspace_bytes(...) bytes, 256-byte aligned.
+ *                    Contents on entry are irrelevant; calls sharing a workspace must not overlap.
+ */
+typedef struct codistill_params {
+  uint64_t struct_bytes;
+  const void* logits;
+  const void* const* peer_logits;
+  const int32_t* labels;
+  const uint8_t* mask;
+  int32_t n;
+  int32_t dtype;
+  int64_t rows;
+  int64_t classes;
+  int64_t row_stride;
+  float alpha;
+  float temperature;
+  float label_smoothing;
+  int32_t dist_kind;
+  int32_t peer_reduce;
+  int32_t reduction;
+  float* row_loss;
+  float* reduced_loss;
+  void* grad_logits;
+  int64_t* counters;
+  int32_t* dev_status;
+  void* workspace;
+  uint64_t workspace_bytes;
+} codistill_params_t;
+
+/*
+ * The objective of Algorithm 1 in the form the paper's experiments use: cross-entropy task
+ * loss, D = MSE on raw logits averaged over the n-1 peers (PAIRWISE_MEAN), no label
+ * smoothing, mean over valid rows, dense rows (row_stride == classes).  `temperature` is
+ * validated (> 0) and otherwise unused because the MSE form has none.
+ * The call draws its scratch from the CUDA stream-ordered allocator (cudaMallocAsync /
+ * cudaFreeAsync on `stream`); use codistill_loss_fwd_bwd_ex to supply the scratch yourself.
+ * `stream` is a cudaStream_t (NULL = default stream).
+ */
+int codistill_loss_fwd_bwd(const void* logits, const void* const* peer_logits /* HOST array */,
+                           const int32_t* labels, const uint8_t* mask, int n, int64_t rows,
+                           int64_t classes, float alpha, float temperature, int dtype,
+                           float* row_loss, float* reduced_loss, void* grad_logits, void* stream);
+
+/* Same operation with every option of codistill_params_t; allocates nothing. */
+int codistill_loss_fwd_bwd_ex(const codistill_params_t* params, void* stream);
+
+/*
+ * Host-buffer variant used for end-to-end use from pageable or pinned HOST memory: every data
+ * pointer in `params` (logits, each peer, labels, mask, row_loss, reduced_loss, grad_logits,
+ * counters, dev_status) is a HOST pointer; params->workspace is a DEVICE buffer of at least
+ * codistill_host_workspace_bytes(...) bytes.  Rows are processed in slices of `chunk_rows`
+ * (0 = library default): host->device copy of a slice, the same kernels as above, device->host
+ * copy of that slice's gradient and losses, software-pipelined over internal streams.  The
+ * call is synchronous: on return every host output is valid.  No arithmetic of the objective
+ * runs on the host.
+ */
+int codistill_loss_fwd_bwd_host(const codistill_params_t* params, int64_t chunk_rows, void* stream);
+
+/* Scratch size for codistill_loss_fwd_bwd_ex (bytes; multiple of 256). */
+size_t codistill_workspace_bytes(int n, int64_t rows, int64_t classes, int dtype);
+
+/* Device scratch size for codistill_loss_fwd_bwd_host with the given slice height. */
+size_t codistill_host_workspace_bytes(int n, int64_t rows, int64_t classes, int dtype, int64_t chunk_rows);
+
+/* Human-readable name of a CODISTILL_ERR_* code (static storage). */
+const char* codistill_status_string(int status);
+
+/* Library version: major * 10000 + minor * 100 + patch. */
+int codistill_version(void);
+
+/*
+ * Name of the kernel regime the dispatcher picks for a problem ("warp", "block" or "tma"), so that
+ * tests and benchmarks can state which kernel they exercised.  Static storage; NULL on bad arguments.
+ */
+const char* codistill_kernel_regime(int n, int64_t rows, int64_t classes, int64_t row_stride, int dtype,
+                                    int dist_kind, int peer_reduce);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* CODISTILL_H_ */
