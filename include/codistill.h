@@ -164,7 +164,8 @@ int codistill_loss_fwd_bwd_host(const codistill_params_t* params, int64_t chunk_
 /* Scratch size for codistill_loss_fwd_bwd_ex (bytes; multiple of 256). */
 size_t codistill_workspace_bytes(int n, int64_t rows, int64_t classes, int dtype);
 
-/* Device scratch size for codistill_loss_fwd_bwd_host with the given slice height. */
+/* Device scratch size for codistill_loss_fwd_bwd_host with the given slice height (0 = default).
+ * Pass the row pitch as `classes` when row_stride > classes. */
 size_t codistill_host_workspace_bytes(int n, int64_t rows, int64_t classes, int dtype, int64_t chunk_rows);
 
 /* Human-readable name of a CODISTILL_ERR_* code (static storage). */
