@@ -36,11 +36,12 @@ FALLBACK_HBM_GBS = 6650.0
 def parse_args():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=50)
+    ap.add_argument("--steps", type=int, default=300)
     ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--workload", type=int, default=4, choices=[1, 2, 3, 4, 5])
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--dist", default="mse", choices=["mse", "kl"])
+    ap.add_argument("--rows", type=int, default=0, help="run a smaller batch of the same recipe (profiling aid)")
     ap.add_argument("--e2e-steps", type=int, default=3)
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
@@ -171,6 +172,8 @@ def run_reference(args):
     if rank != 0:
         return
     w = synth.WORKLOADS[args.workload]
+    if args.rows:
+        w = synth.scaled(w, rows=args.rows)
     steps, warmup = max(1, args.steps), max(0, args.warmup)
     value, dt, rows, cores = time_oracle(w, args.dist, steps, warmup)
     sample = f"first {rows} rows of the workload per step, all {w.n} models, fp64 oracle as it stands"
@@ -236,6 +239,8 @@ def run_ours(args):
     cb.load_library()
 
     w0 = synth.WORKLOADS[args.workload]
+    if args.rows:
+        w0 = synth.scaled(w0, rows=args.rows)
     dist_code = cb.DIST_KL_SOFTMAX if args.dist == "kl" else cb.DIST_MSE_LOGITS
     w, models, labels, mask = make_device_inputs(w0, torch, seed_offset=rank)   # each rank: its own batch
     plan = cb.Plan(models[0], models[1:], labels, mask, alpha=w.alpha, temperature=w.temperature,
