@@ -49,7 +49,8 @@ enum {
   CODISTILL_ERR_PARAM = 4,       /* temperature <= 0, non-finite alpha, label_smoothing outside [0,1), bad enum */
   CODISTILL_ERR_UNSUPPORTED = 5, /* valid request this build cannot serve (e.g. n - 1 > CODISTILL_MAX_PEERS) */
   CODISTILL_ERR_CUDA = 6,        /* a CUDA runtime call failed; the CUDA error is left for cudaGetLastError */
-  CODISTILL_ERR_WORKSPACE = 7    /* workspace NULL, misaligned (256 B) or smaller than codistill_workspace_bytes */
+  CODISTILL_ERR_WORKSPACE = 7,   /* workspace NULL, misaligned (256 B) or smaller than codistill_workspace_bytes */
+  CODISTILL_ERR_TOO_LARGE = 8    /* codistill_loss_fwd_bwd_static only: rows > CODISTILL_STATIC_MAX_ROWS */
 };
 
 /* element type of logits, peers and grad_logits */
@@ -145,6 +146,40 @@ int codistill_loss_fwd_bwd(const void* logits, const void* const* peer_logits /*
                            const int32_t* labels, const uint8_t* mask, int n, int64_t rows,
                            int64_t classes, float alpha, float temperature, int dtype,
                            float* row_loss, float* reduced_loss, void* grad_logits, void* stream);
+
+/*
+ * Allocation-free form of codistill_loss_fwd_bwd.  (The paper has no counterpart for this entry
+ * point; it exists for deployment reasons only.)
+ *
+ * Who needs it: programs that must not touch a CUDA allocator when they call the loss.  Typical
+ * cases are a serving or training process whose framework claimed all device memory at start-up,
+ * so that a later cudaMalloc / cudaMallocAsync fails or stalls, and latency-critical loops that ban
+ * allocator calls because those may synchronise the device.  The basic entry point above takes its
+ * scratch from the stream-ordered allocator and the _ex form expects the caller to have allocated
+ * a workspace; this one needs neither.
+ *
+ * How: the scratch (row-validity counts, per-row flag words, the completion ticket) lives in a
+ * fixed array inside the library's device image.  Every GPU that loads the library holds that
+ * array (about 0.5 MiB) until the process exits.  The array is sized for at most
+ * CODISTILL_STATIC_MAX_ROWS rows; a larger `rows` returns CODISTILL_ERR_TOO_LARGE and launches
+ * nothing.  The call performs no cudaMalloc, cudaFree or other allocating routine.
+ *
+ * Arguments, defaults and outputs are exactly those of codistill_loss_fwd_bwd, except that
+ * row_loss must not be NULL (a missing row_loss would need per-row scratch of the caller's size).
+ *
+ * Set-up: the first call on each device looks up the device address of the array (the device
+ * must be current, as for every call).  Make that first call outside any stream capture.
+ *
+ * Sharing: all calls on a device use the same array, which keeps whatever the previous call left
+ * in it; each call clears the words that must start at zero before using them.  Two calls that
+ * overlap on the GPU (different streams, no ordering between them) race on the array and give
+ * wrong results: order them, or use codistill_loss_fwd_bwd_ex with separate workspaces.
+ */
+#define CODISTILL_STATIC_MAX_ROWS 65536
+int codistill_loss_fwd_bwd_static(const void* logits, const void* const* peer_logits /* HOST array */,
+                                  const int32_t* labels, const uint8_t* mask, int n, int64_t rows,
+                                  int64_t classes, float alpha, float temperature, int dtype,
+                                  float* row_loss, float* reduced_loss, void* grad_logits, void* stream);
 
 /* Same operation with every option of codistill_params_t; allocates nothing. */
 int codistill_loss_fwd_bwd_ex(const codistill_params_t* params, void* stream);

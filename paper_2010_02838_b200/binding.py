@@ -22,9 +22,12 @@ PEERS_PAIRWISE_MEAN, PEERS_MEAN_TARGET = 0, 1
 REDUCE_MEAN_VALID, REDUCE_SUM = 0, 1
 DEV_BAD_LABEL, DEV_TIMEOUT, DEV_ASSERT = 1, 2, 4
 MAX_PEERS = 31
+STATIC_MAX_ROWS = 65536
+ERR_TOO_LARGE = 8
 
 EXPORTS = (
     "codistill_loss_fwd_bwd", "codistill_loss_fwd_bwd_ex", "codistill_loss_fwd_bwd_host",
+    "codistill_loss_fwd_bwd_static",
     "codistill_workspace_bytes", "codistill_host_workspace_bytes", "codistill_status_string",
     "codistill_version", "codistill_kernel_regime",
 )
@@ -81,6 +84,8 @@ def load_library() -> ctypes.CDLL:
     vp, i64, i32, f32 = ctypes.c_void_p, ctypes.c_int64, ctypes.c_int, ctypes.c_float
     lib.codistill_loss_fwd_bwd.restype = i32
     lib.codistill_loss_fwd_bwd.argtypes = [vp, ctypes.POINTER(vp), vp, vp, i32, i64, i64, f32, f32, i32, vp, vp, vp, vp]
+    lib.codistill_loss_fwd_bwd_static.restype = i32
+    lib.codistill_loss_fwd_bwd_static.argtypes = lib.codistill_loss_fwd_bwd.argtypes
     lib.codistill_loss_fwd_bwd_ex.restype = i32
     lib.codistill_loss_fwd_bwd_ex.argtypes = [ctypes.POINTER(Params), vp]
     lib.codistill_loss_fwd_bwd_host.restype = i32
@@ -191,6 +196,29 @@ def codistill_loss_fwd_bwd(logits: torch.Tensor, peer_logits, labels: torch.Tens
     rc = lib.codistill_loss_fwd_bwd(_ptr(logits), ptrs, _ptr(labels), _ptr(mask), len(peers) + 1, rows, C,
                                     float(alpha), float(temperature), dtype_code(logits.dtype),
                                     _ptr(out.row_loss), _ptr(out.loss), _ptr(out.grad), _stream_ptr(stream))
+    if rc != OK:
+        raise CodistillError(rc)
+    return out
+
+
+def codistill_loss_fwd_bwd_static(logits: torch.Tensor, peer_logits, labels: torch.Tensor,
+                                  mask: torch.Tensor | None, out: Outputs, *, alpha: float = 1.0,
+                                  temperature: float = 1.0, stream: torch.cuda.Stream | None = None) -> Outputs:
+    """The allocation-free entry point of the C ABI.  For callers that must not touch a CUDA
+    allocator at call time (all device memory already claimed by a framework, or a loop that bans
+    allocator calls): the library's scratch is a fixed array in its device image, good for at most
+    ``STATIC_MAX_ROWS`` rows.  Nothing is allocated here either, so ``out`` (row_loss, loss and
+    optionally grad) must be supplied.  Calls on one device share the scratch: keep them ordered."""
+    lib = load_library()
+    peers = list(peer_logits)
+    _require_cuda(logits, labels, mask, out.row_loss, out.loss, out.grad, *peers)
+    rows, stride, C = _check_shapes(logits, peers, labels, mask, None)
+    if rows > 1 and stride != C:
+        raise ValueError("the allocation-free call needs dense rows")
+    ptrs = (ctypes.c_void_p * max(1, len(peers)))(*[p.data_ptr() for p in peers])
+    rc = lib.codistill_loss_fwd_bwd_static(_ptr(logits), ptrs, _ptr(labels), _ptr(mask), len(peers) + 1, rows, C,
+                                           float(alpha), float(temperature), dtype_code(logits.dtype),
+                                           _ptr(out.row_loss), _ptr(out.loss), _ptr(out.grad), _stream_ptr(stream))
     if rc != OK:
         raise CodistillError(rc)
     return out

@@ -341,6 +341,7 @@ const char* codistill_status_string(int status) {
     case CODISTILL_ERR_UNSUPPORTED: return "request not supported by this build";
     case CODISTILL_ERR_CUDA: return "a CUDA runtime call failed";
     case CODISTILL_ERR_WORKSPACE: return "workspace missing, misaligned or too small";
+    case CODISTILL_ERR_TOO_LARGE: return "rows exceed CODISTILL_STATIC_MAX_ROWS, the capacity of the built-in scratch";
     default: return "unknown status";
   }
 }
@@ -431,3 +432,65 @@ const char* codistill_kernel_regime(int n, int64_t rows, int64_t classes, int64_
 }
 
 }  // extern "C"
+
+// ------------------------------------------------------------------ allocation-free entry point
+// Scratch of codistill_loss_fwd_bwd_static: one workspace for up to CODISTILL_STATIC_MAX_ROWS rows,
+// part of the device image of this library (each GPU that loads it keeps the array until exit).
+// In host code `g_static_scratch` is only a handle for cudaGetSymbolAddress, never a device address.
+namespace codistill {
+constexpr size_t kStaticScratchBytes = 256 + 1024 + 2 * 4 * (size_t)CODISTILL_STATIC_MAX_ROWS;
+static __device__ __align__(256) unsigned char g_static_scratch[kStaticScratchBytes];
+
+// Device address of the scratch array on the current device, looked up once per device.
+static int static_scratch_address(void** out) {
+  static void* cache[64];
+  static bool known[64];
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess) return CODISTILL_ERR_CUDA;
+  if (dev >= 0 && dev < 64 && known[dev]) { *out = cache[dev]; return CODISTILL_OK; }
+  void* ptr = nullptr;
+  if (cudaGetSymbolAddress(&ptr, g_static_scratch) != cudaSuccess || ptr == nullptr) return CODISTILL_ERR_CUDA;
+  if (dev >= 0 && dev < 64) { cache[dev] = ptr; known[dev] = true; }
+  *out = ptr;
+  return CODISTILL_OK;
+}
+}  // namespace codistill
+
+extern "C" int codistill_loss_fwd_bwd_static(const void* logits, const void* const* peer_logits, const int32_t* labels,
+                                             const uint8_t* mask, int n, int64_t rows, int64_t classes, float alpha,
+                                             float temperature, int dtype, float* row_loss, float* reduced_loss,
+                                             void* grad_logits, void* stream) {
+  using namespace codistill;
+  codistill_params_t p;
+  memset(&p, 0, sizeof(p));
+  p.struct_bytes = sizeof(p);
+  p.logits = logits;
+  p.peer_logits = peer_logits;
+  p.labels = labels;
+  p.mask = mask;
+  p.n = n;
+  p.dtype = dtype;
+  p.rows = rows;
+  p.classes = classes;
+  p.row_stride = classes;
+  p.alpha = alpha;
+  p.temperature = temperature;
+  p.dist_kind = CODISTILL_DIST_MSE_LOGITS;
+  p.peer_reduce = CODISTILL_PEERS_PAIRWISE_MEAN;
+  p.reduction = CODISTILL_REDUCE_MEAN_VALID;
+  p.row_loss = row_loss;
+  p.reduced_loss = reduced_loss;
+  p.grad_logits = grad_logits;
+  p.workspace = reinterpret_cast<void*>(uintptr_t(256));  // placeholder for validation; replaced below
+  const int v = validate(&p, false);
+  if (v != CODISTILL_OK) return v;
+  if (row_loss == nullptr) return CODISTILL_ERR_NULL;
+  if (rows > (int64_t)CODISTILL_STATIC_MAX_ROWS) return CODISTILL_ERR_TOO_LARGE;
+  if (ws_layout(rows).total > kStaticScratchBytes) return CODISTILL_ERR_TOO_LARGE;
+  void* scratch = nullptr;
+  const int rc = static_scratch_address(&scratch);
+  if (rc != CODISTILL_OK) return rc;
+  p.workspace = scratch;
+  p.workspace_bytes = kStaticScratchBytes;
+  return run_device(&p, static_cast<cudaStream_t>(stream));
+}
