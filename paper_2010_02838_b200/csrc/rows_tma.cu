@@ -1,48 +1,45 @@
 // Persistent, warp-specialised kernel for long rows ("tma" regime), MSE-on-logits distance.
 //
-// One CTA per SM.  Warp 0 is the producer: it draws row ids from a global counter and moves row
-// images from HBM into shared memory with 1-D bulk asynchronous copies (cp.async.bulk) that
-// complete on mbarriers.  The own row of a model stays resident in one of one or two row
-// buffers; the n-1 peer rows are streamed chunk by chunk (chunk-major: chunk k of peer 0, 1, ...,
-// then chunk k+1) through a ring of 16 KiB stages.  The 16 consumer warps make one pass over the
-// resident own row for the softmax statistics, then consume the ring: per 16-byte segment they
-// accumulate sum_j (z - z_j) and sum_j (z - z_j)^2, track what the arg-max agreement needs, and
-// write the gradient with 128-bit stores.  Every logit is read from HBM exactly once and the
-// gradient is written once.
+// Each CTA owns one resident row buffer and a ring of stages; as many CTAs as fit run per SM (two
+// for 64 KiB rows), so that one CTA's statistics pass overlaps the other's streaming pass.
+//   warp 0  scheduler + own-row producer: draws row ids from a global counter (mask byte and label
+//           are fetched one row ahead), publishes them in a small ring of row-info slots, and moves
+//           the own row image into the row buffer piece by piece with 1-D bulk asynchronous copies
+//           (cp.async.bulk, no multicast) that complete on one mbarrier per piece.  A piece is
+//           refilled for the next row as soon as the consumers are done with it, so the next own
+//           row streams in behind the current row's second pass.
+//   warp 1  peer producer: streams the n-1 peer rows chunk by chunk (chunk-major: chunk k of peer
+//           0, 1, ..., then chunk k+1) through the ring of stages.
+//   others  consumers: first pass over the resident own row (max, sum exp, sum z, first arg-max),
+//           then per chunk: consume the peers from the ring (sum_j (z - z_j), sum_j (z - z_j)^2,
+//           what the arg-max agreement needs), write the gradient with 128-bit stores, release the
+//           own piece.
+// Every logit is read from HBM exactly once and the gradient is written once.
 //
 // A "row image" is the 16-byte aligned byte range that contains the row: rows whose byte length
 // is not a multiple of 16 start at varying offsets `head` inside their first segment.  Segments
-// that are only partly inside the row ("edge" segments) take a masked slow path.
+// that are only partly inside the row ("edge" segments) take a masked slow path.  Every valid row
+// uses the same number of pieces (some possibly empty), so that barrier phases advance uniformly.
 #include "common.cuh"
 
 namespace codistill {
 
-// Tuning constants (overridable at compile time for experiments).
-#ifndef CODISTILL_TMA_CONSUMER_WARPS
-#define CODISTILL_TMA_CONSUMER_WARPS 16
-#endif
-#ifndef CODISTILL_TMA_CTAS_PER_SM
-#define CODISTILL_TMA_CTAS_PER_SM 1
-#endif
-#ifndef CODISTILL_TMA_CHUNK_BYTES
-#define CODISTILL_TMA_CHUNK_BYTES 16384
-#endif
-constexpr int kConsumerWarps = CODISTILL_TMA_CONSUMER_WARPS;
-constexpr int kCtasPerSm = CODISTILL_TMA_CTAS_PER_SM;
-constexpr int kConsumers = kConsumerWarps * 32;
-constexpr int kTmaThreads = kConsumers + 32;
-constexpr int kChunkBytes = CODISTILL_TMA_CHUNK_BYTES;
-constexpr int kSegPerChunk = kChunkBytes / 16;
-constexpr int kSegPerThread = kSegPerChunk / kConsumers;
-static_assert(kSegPerThread * kConsumers == kSegPerChunk, "a chunk splits evenly over the consumer threads");
 constexpr int kMaxStages = 12;
-constexpr int kCtrlBytes = 4096;
-constexpr int kOwnPieceBytes = 32768;
+constexpr int kMaxPieces = 32;
+constexpr int kInfoSlots = 4;
+constexpr int kCtrlBytes = 5120;
+constexpr int kProducerThreads = 64;   // warp 0: scheduler + own row, warp 1: peers
+constexpr int kSegPerThread = 2;       // 16-byte segments per consumer thread per chunk
+constexpr int kMaxConsumerWarps = 16;
+constexpr uint32_t kBulkPieceBytes = 32768;
 constexpr unsigned long long kWaitLimitNs = 2000000000ull;  // bounded waits: 2 s, then CODISTILL_DEV_TIMEOUT
 
 struct TmaCfg {
-  int own_bufs;
-  int stages;
+  int consumer_warps;  // 8 (two CTAs per SM) or 16 (one CTA per SM)
+  int ctas_per_sm;
+  int stages;          // ring stages of chunk_bytes each
+  int pieces;          // chunks per row image (same for every row of the call)
+  uint32_t chunk_bytes;
   uint32_t own_buf_bytes;
   uint32_t smem_bytes;
 };
@@ -54,14 +51,16 @@ struct RowInfo {
 };
 
 struct Ctrl {  // lives at the start of dynamic shared memory
-  uint64_t own_full[2];
-  uint64_t own_empty[2];
+  uint64_t own_full[kMaxPieces];
+  uint64_t own_empty[kMaxPieces];
   uint64_t ring_full[kMaxStages];
   uint64_t ring_empty[kMaxStages];
-  RowInfo info[2];
+  uint64_t info_full[kInfoSlots];
+  uint64_t info_empty[kInfoSlots];
+  RowInfo info[kInfoSlots];
   int abort_flag;
   int last_flag;
-  float red[2][kConsumerWarps * 24];  // reduction scratch of the consumers, two alternating halves
+  float red[2][kMaxConsumerWarps * 24];  // reduction scratch of the consumers, two alternating halves
   double fin[32];
 };
 static_assert(sizeof(Ctrl) <= kCtrlBytes, "control block fits its slot");
@@ -100,7 +99,6 @@ __device__ __forceinline__ unsigned long long global_timer_ns() {
   asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
   return t;
 }
-__device__ __forceinline__ void consumer_bar() { asm volatile("bar.sync 1, %0;" ::"n"(kConsumers) : "memory"); }
 
 // Wait for a phase of an mbarrier, but never for ever: after kWaitLimitNs the CTA-wide abort flag
 // and the device status are set and every later wait returns at once (results are then invalid).
@@ -221,22 +219,32 @@ __device__ __forceinline__ RowGeom row_geom(int64_t local_row, int64_t row_strid
   return g;
 }
 
-// Block reductions among the 512 consumer threads (one named barrier each).
+// Geometry shared by every row of a call: segments of the longest row image.
+template <typename T>
+__host__ __device__ inline int64_t max_row_segments(int64_t row_stride, int64_t classes) {
+  constexpr int V = 16 / (int)sizeof(T);
+  const int64_t head_max = (row_stride % V == 0) ? 0 : V - 1;
+  return (head_max + classes + V - 1) / V;
+}
+
+// Block reductions among the NCW * 32 consumer threads (one named barrier each).
+template <int NCW>
 struct ConsumerReduce {
   Ctrl* ctrl;
   int toggle;
-  int warp, lane;  // consumer warp index 0..15
+  int warp, lane;  // consumer warp index 0..NCW-1
+  __device__ __forceinline__ static void bar() { asm volatile("bar.sync 1, %0;" ::"n"(NCW * 32) : "memory"); }
   template <int N>
   __device__ __forceinline__ void sum(float (&v)[N]) {
     float* s = ctrl->red[toggle];
 #pragma unroll
     for (int k = 0; k < N; ++k) {
       v[k] = warp_sum(v[k]);
-      if (lane == 0) s[k * kConsumerWarps + warp] = v[k];
+      if (lane == 0) s[k * NCW + warp] = v[k];
     }
-    consumer_bar();
+    bar();
 #pragma unroll
-    for (int k = 0; k < N; ++k) v[k] = warp_sum(lane < kConsumerWarps ? s[k * kConsumerWarps + lane] : 0.f);
+    for (int k = 0; k < N; ++k) v[k] = warp_sum(lane < NCW ? s[k * NCW + lane] : 0.f);
     toggle ^= 1;
   }
   template <int N>
@@ -245,11 +253,11 @@ struct ConsumerReduce {
 #pragma unroll
     for (int k = 0; k < N; ++k) {
       v[k] = warp_max(v[k]);
-      if (lane == 0) s[k * kConsumerWarps + warp] = v[k];
+      if (lane == 0) s[k * NCW + warp] = v[k];
     }
-    consumer_bar();
+    bar();
 #pragma unroll
-    for (int k = 0; k < N; ++k) v[k] = warp_max(lane < kConsumerWarps ? s[k * kConsumerWarps + lane] : -INFINITY);
+    for (int k = 0; k < N; ++k) v[k] = warp_max(lane < NCW ? s[k * NCW + lane] : -INFINITY);
     toggle ^= 1;
   }
   __device__ __forceinline__ int min_int(int v) {
@@ -257,8 +265,8 @@ struct ConsumerReduce {
 #pragma unroll
     for (int o = 16; o > 0; o >>= 1) v = ::min(v, __shfl_xor_sync(0xffffffffu, v, o));
     if (lane == 0) s[warp] = v;
-    consumer_bar();
-    v = lane < kConsumerWarps ? s[lane] : 0x7fffffff;
+    bar();
+    v = lane < NCW ? s[lane] : 0x7fffffff;
 #pragma unroll
     for (int o = 16; o > 0; o >>= 1) v = ::min(v, __shfl_xor_sync(0xffffffffu, v, o));
     toggle ^= 1;
@@ -267,29 +275,49 @@ struct ConsumerReduce {
 };
 
 // ------------------------------------------------------------------ producer helpers
-// Moves `img_bytes` of a row image from `src` (16-byte aligned) to `dst`, completing on `bar`.
-// `tma_bytes` <= img_bytes is the part that may be read as whole segments; the elements between
-// tma_bytes and valid_end (a partial last segment at the very end of a tensor) are fetched with
-// plain loads by the lanes of the producer warp.  Called by the whole producer warp.
+// Moves bytes [begin, end) of a row image whose start is `src` (16-byte aligned) to `dst` (the
+// shared-memory address of byte `begin`), completing on `bar` (one arrival + the byte count).
+// `tma_limit` is where whole-segment reads must stop: the elements between tma_limit and valid_end
+// (a partial last segment at the very end of a tensor) are fetched with plain loads by the lanes of
+// the producer warp.  Called by a whole producer warp.
 template <typename T>
 __device__ __forceinline__ void produce_copy(char* dst, const char* src, uint32_t begin, uint32_t end, uint32_t tma_limit,
                                              uint32_t valid_end, uint64_t* bar, int lane) {
-  // [begin, end) is the byte range of the image handled by this copy
   const uint32_t tma_end = end < tma_limit ? end : tma_limit;
   if (end > tma_limit) {  // partial last segment that must not be read as a whole
     const uint32_t first = tma_limit > begin ? tma_limit : begin;
     const uint32_t off = first + (uint32_t)lane * (uint32_t)sizeof(T);
-    if (off < valid_end) *reinterpret_cast<T*>(dst + (off - begin)) = *reinterpret_cast<const T*>(src + off);
+    if (off < valid_end && off < end) *reinterpret_cast<T*>(dst + (off - begin)) = *reinterpret_cast<const T*>(src + off);
     __syncwarp();
   }
   if (lane == 0) {
     const uint32_t bytes = tma_end > begin ? tma_end - begin : 0u;
     mbar_arrive_expect_tx(bar, bytes);
-    for (uint32_t o = 0; o < bytes; o += kOwnPieceBytes) {
-      const uint32_t piece = bytes - o < (uint32_t)kOwnPieceBytes ? bytes - o : (uint32_t)kOwnPieceBytes;
+    for (uint32_t o = 0; o < bytes; o += kBulkPieceBytes) {
+      const uint32_t piece = bytes - o < kBulkPieceBytes ? bytes - o : kBulkPieceBytes;
       bulk_g2s(dst + o, src + begin + o, piece, bar);
     }
   }
+}
+
+// Per-row quantities both producers derive from the row id.
+struct RowCopy {
+  uint32_t img_bytes, valid_end, tma_limit;
+  int64_t row_off;  // image start relative to the tensor, in bytes
+};
+template <typename T>
+__device__ __forceinline__ RowCopy row_copy(const KArgs& a, long long r) {
+  constexpr int ES = (int)sizeof(T);
+  const int64_t lr = r - a.row_begin;
+  const RowGeom g = row_geom<T>(lr, a.row_stride, a.classes);
+  RowCopy c;
+  c.img_bytes = (uint32_t)g.n_seg * 16u;
+  c.valid_end = (uint32_t)(g.head + a.classes) * ES;
+  // The last row of the whole call may end inside a segment that reaches past the tensor.
+  const bool clip = (r == a.rows_total - 1) && ((a.row_stride - a.classes) * ES < 16) && (c.valid_end & 15u);
+  c.tma_limit = clip ? (c.valid_end & ~15u) : c.img_bytes;
+  c.row_off = lr * a.row_stride * ES - (int64_t)g.head * ES;
+  return c;
 }
 
 // First column of segment `s` whose value equals m, or INT_MAX.
@@ -344,25 +372,32 @@ __device__ __noinline__ SlowPeer<T> slow_peer(SegPairs<T> zs, uint4 raw, int seg
 }
 
 // ------------------------------------------------------------------ the kernel
-template <typename T, int P, bool PW>
-__global__ void __launch_bounds__(kTmaThreads, kCtasPerSm) rows_tma_kernel(const __grid_constant__ KArgs a, const TmaCfg cfg) {
+// T: element type; P: number of peers (compile time); PW: the loss sums squared pairwise differences
+// (otherwise the squared difference to the averaged peer); NCW: consumer warps per CTA.
+template <typename T, int P, bool PW, int NCW>
+__global__ void __launch_bounds__(NCW * 32 + kProducerThreads, NCW == 8 ? 2 : 1)
+rows_tma_kernel(const __grid_constant__ KArgs a, const TmaCfg cfg) {
   constexpr int V = SegOps<T>::V;
   constexpr int H = SegOps<T>::H;
   constexpr int PD = P > 0 ? P : 1;
   constexpr int ES = (int)sizeof(T);
+  constexpr int kConsumers = NCW * 32;
+  constexpr int kSegPerChunk = kConsumers * kSegPerThread;
+  constexpr uint32_t kChunkBytes = kSegPerChunk * 16;
   extern __shared__ __align__(128) unsigned char smem_raw[];
   Ctrl* ctrl = reinterpret_cast<Ctrl*>(smem_raw);
-  char* own_base = reinterpret_cast<char*>(smem_raw) + kCtrlBytes;
-  char* ring_base = own_base + (size_t)cfg.own_bufs * cfg.own_buf_bytes;
+  char* own_buf = reinterpret_cast<char*>(smem_raw) + kCtrlBytes;
+  char* ring_base = own_buf + cfg.own_buf_bytes;
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  const int n_own = cfg.own_bufs, n_stage = cfg.stages;
+  const int n_stage = cfg.stages, n_pieces = cfg.pieces;
   const int64_t C = a.classes;
   const bool with_term = (P >= 1 && a.alpha != 0.f);
   const bool stream_peers = (P >= 1) && (with_term || a.want_flags);
 
   if (threadIdx.x == 0) {
-    for (int b = 0; b < 2; ++b) { mbar_init(&ctrl->own_full[b], 1); mbar_init(&ctrl->own_empty[b], kConsumerWarps); }
-    for (int s = 0; s < kMaxStages; ++s) { mbar_init(&ctrl->ring_full[s], 1); mbar_init(&ctrl->ring_empty[s], kConsumerWarps); }
+    for (int k = 0; k < kMaxPieces; ++k) { mbar_init(&ctrl->own_full[k], 1); mbar_init(&ctrl->own_empty[k], NCW); }
+    for (int s = 0; s < kMaxStages; ++s) { mbar_init(&ctrl->ring_full[s], 1); mbar_init(&ctrl->ring_empty[s], NCW); }
+    for (int s = 0; s < kInfoSlots; ++s) { mbar_init(&ctrl->info_full[s], 1); mbar_init(&ctrl->info_empty[s], NCW + 1); }
     ctrl->abort_flag = 0;
     ctrl->last_flag = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -370,9 +405,7 @@ __global__ void __launch_bounds__(kTmaThreads, kCtasPerSm) rows_tma_kernel(const
   __syncthreads();
 
   if (warp == 0) {
-    // ============================== producer warp ==============================
-    uint32_t q = 0;  // ring items issued so far
-    int last_it[2] = {-1, -1};
+    // ============================== scheduler + own-row producer ==============================
     // Row ids come from a global counter.  The counter and the row's mask byte and label are fetched
     // two and one iterations ahead (lane 0), so that their latency never sits between two rows.
     long long t_next = 0, t_next2 = 0;
@@ -382,6 +415,7 @@ __global__ void __launch_bounds__(kTmaThreads, kCtasPerSm) rows_tma_kernel(const
       t_next2 = a.row_begin + (long long)atomicAdd(&a.hdr->next_row, 1u);
       if (t_next < a.row_end) { mask_next = a.mask ? a.mask[t_next] : 1; label_next = a.labels[t_next]; }
     }
+    int v = 0;  // valid rows copied so far
     for (int it = 0;; ++it) {
       long long r = t_next;
       int mask_v = mask_next, label_v = label_next;
@@ -393,61 +427,66 @@ __global__ void __launch_bounds__(kTmaThreads, kCtasPerSm) rows_tma_kernel(const
       r = __shfl_sync(0xffffffffu, r, 0);
       mask_v = __shfl_sync(0xffffffffu, mask_v, 0);
       label_v = __shfl_sync(0xffffffffu, label_v, 0);
-      const int b = it % n_own;
       const bool more = r < a.row_end;
       const bool valid = more && mask_v != 0 && label_v >= 0 && (int64_t)label_v < C;
-      const int64_t lr = r - a.row_begin;
-      const RowGeom g = row_geom<T>(valid ? lr : 0, a.row_stride, C);
-      const uint32_t img_bytes = (uint32_t)g.n_seg * 16u;
-      const uint32_t valid_end = (uint32_t)(g.head + C) * ES;
-      // The last row of the whole call may end inside a segment that reaches past the tensor.
-      const bool clip = (r == a.rows_total - 1) && ((a.row_stride - C) * ES < 16) && (valid_end & 15u);
-      const uint32_t tma_limit = clip ? (valid_end & ~15u) : img_bytes;
-      const int64_t row_off = lr * a.row_stride * ES - (int64_t)g.head * ES;  // image start relative to the tensor
-      const int n_items = (valid && stream_peers) ? ((g.n_seg + kSegPerChunk - 1) / kSegPerChunk) * P : 0;
-      auto issue_item = [&](int idx) {
-        const int k = idx / PD, j = idx - k * PD;
-        const uint32_t begin = (uint32_t)k * kChunkBytes;
-        const uint32_t end = begin + kChunkBytes < img_bytes ? begin + kChunkBytes : img_bytes;
-        const int s = q % n_stage;
-        if (q >= (uint32_t)n_stage) wait_bounded(&ctrl->ring_empty[s], ((q / n_stage) - 1) & 1, ctrl, a.hdr);
-        produce_copy<T>(ring_base + (size_t)s * kChunkBytes, reinterpret_cast<const char*>(a.peers[j]) + row_off, begin, end,
-                        tma_limit, valid_end, &ctrl->ring_full[s], lane);
-        ++q;
-      };
-      // With a single row buffer the next own row cannot be fetched before the current row is
-      // finished; fill the ring with the next row's first peer chunks meanwhile.  Never more than
-      // the ring holds, or the producer would wait for stages the consumers cannot yet free.
-      const int pre = (n_own == 1) ? (n_items < n_stage ? n_items : n_stage) : 0;
-      for (int idx = 0; idx < pre; ++idx) issue_item(idx);
-      if (it >= n_own) wait_bounded(&ctrl->own_empty[b], ((it / n_own) - 1) & 1, ctrl, a.hdr);
-      last_it[b] = it;
+      const int slot = it % kInfoSlots;
+      if (it >= kInfoSlots) wait_bounded(&ctrl->info_empty[slot], ((it / kInfoSlots) - 1) & 1, ctrl, a.hdr);
       if (lane == 0) {
-        ctrl->info[b].row = more ? r : -1;
-        ctrl->info[b].valid = valid;
-        ctrl->info[b].label = label_v;
+        ctrl->info[slot].row = more ? r : -1;
+        ctrl->info[slot].valid = valid;
+        ctrl->info[slot].label = label_v;
+        mbar_arrive(&ctrl->info_full[slot]);
       }
-      if (!valid) {
-        __syncwarp();
-        if (lane == 0) mbar_arrive(&ctrl->own_full[b]);
-        if (!more) break;
-        continue;
+      if (!more) break;
+      if (!valid) continue;
+      const RowCopy rc = row_copy<T>(a, r);
+      const char* src = reinterpret_cast<const char*>(a.own) + rc.row_off;
+      for (int k = 0; k < n_pieces; ++k) {
+        if (v >= 1) wait_bounded(&ctrl->own_empty[k], (v - 1) & 1, ctrl, a.hdr);
+        const uint32_t begin = (uint32_t)k * kChunkBytes;
+        uint32_t end = begin + kChunkBytes < rc.img_bytes ? begin + kChunkBytes : rc.img_bytes;
+        if (end < begin) end = begin;  // empty piece of a shorter row image
+        produce_copy<T>(own_buf + begin, src, begin, end, rc.tma_limit, rc.valid_end, &ctrl->own_full[k], lane);
       }
-      produce_copy<T>(own_base + (size_t)b * cfg.own_buf_bytes, reinterpret_cast<const char*>(a.own) + row_off, 0u, img_bytes,
-                      tma_limit, valid_end, &ctrl->own_full[b], lane);
-      for (int idx = pre; idx < n_items; ++idx) issue_item(idx);
+      ++v;
     }
     // Before leaving, make sure no copy armed by this warp is still in flight (bounded).
-    for (int b = 0; b < n_own; ++b)
-      if (last_it[b] >= 0) wait_bounded(&ctrl->own_full[b], (last_it[b] / n_own) & 1, ctrl, a.hdr);
+    if (v >= 1)
+      for (int k = 0; k < n_pieces; ++k) wait_bounded(&ctrl->own_full[k], (v - 1) & 1, ctrl, a.hdr);
+  } else if (warp == 1) {
+    // ============================== peer producer ==============================
+    uint32_t q = 0;  // ring items issued so far
+    for (int it = 0;; ++it) {
+      const int slot = it % kInfoSlots;
+      wait_bounded(&ctrl->info_full[slot], (it / kInfoSlots) & 1, ctrl, a.hdr);
+      const long long r = ctrl->info[slot].row;
+      const bool valid = ctrl->info[slot].valid != 0;
+      __syncwarp();
+      if (lane == 0) mbar_arrive(&ctrl->info_empty[slot]);
+      if (r < 0) break;
+      if (!valid || !stream_peers) continue;
+      const RowCopy rc = row_copy<T>(a, r);
+      for (int k = 0; k < n_pieces; ++k) {
+        const uint32_t begin = (uint32_t)k * kChunkBytes;
+        uint32_t end = begin + kChunkBytes < rc.img_bytes ? begin + kChunkBytes : rc.img_bytes;
+        if (end < begin) end = begin;
+#pragma unroll 1
+        for (int j = 0; j < P; ++j, ++q) {
+          const int s = q % n_stage;
+          if (q >= (uint32_t)n_stage) wait_bounded(&ctrl->ring_empty[s], ((q / n_stage) - 1) & 1, ctrl, a.hdr);
+          produce_copy<T>(ring_base + (size_t)s * kChunkBytes, reinterpret_cast<const char*>(a.peers[j]) + rc.row_off, begin, end,
+                          rc.tma_limit, rc.valid_end, &ctrl->ring_full[s], lane);
+        }
+      }
+    }
     for (uint32_t i = 0; i < (uint32_t)n_stage && i < q; ++i) {
       const uint32_t qi = q - 1 - i;
       wait_bounded(&ctrl->ring_full[qi % n_stage], (qi / n_stage) & 1, ctrl, a.hdr);
     }
   } else {
     // ============================== consumer warps ==============================
-    const int tid = threadIdx.x - 32;
-    ConsumerReduce red{ctrl, 0, warp - 1, lane};
+    const int tid = threadIdx.x - kProducerThreads;
+    ConsumerReduce<NCW> red{ctrl, 0, warp - 2, lane};
     float w = 1.f;
     if (a.reduction == CODISTILL_REDUCE_MEAN_VALID) {
       const int64_t nv = total_valid(a);
@@ -455,19 +494,22 @@ __global__ void __launch_bounds__(kTmaThreads, kCtasPerSm) rows_tma_kernel(const
     }
     const float inv_P = P >= 1 ? 1.f / (float)P : 0.f;
     uint32_t q = 0;
+    int v = 0;  // valid rows processed so far
     for (int it = 0;; ++it) {
-      const int b = it % n_own;
-      wait_bounded(&ctrl->own_full[b], (it / n_own) & 1, ctrl, a.hdr);
-      const long long r = ctrl->info[b].row;
+      const int slot = it % kInfoSlots;
+      wait_bounded(&ctrl->info_full[slot], (it / kInfoSlots) & 1, ctrl, a.hdr);
+      const long long r = ctrl->info[slot].row;
+      const bool valid = ctrl->info[slot].valid != 0;
+      const int y = ctrl->info[slot].label;
+      __syncwarp();
+      if (lane == 0) mbar_arrive(&ctrl->info_empty[slot]);
       if (r < 0) break;
-      const bool valid = ctrl->info[b].valid != 0;
-      const int y = ctrl->info[b].label;
       const int64_t lr = r - a.row_begin;
       const RowGeom g = row_geom<T>(lr, a.row_stride, C);
-      const char* img = own_base + (size_t)b * cfg.own_buf_bytes;
+      const char* img = own_buf;
       char* g_img = a.grad ? reinterpret_cast<char*>(a.grad) + lr * a.row_stride * ES - (int64_t)g.head * ES : nullptr;
 
-      if (!valid) {
+      if (!valid) {  // masked row: zero gradient, no loss, no counts; nothing was copied for it
         if (g_img) {
           for (int s = tid; s < g.n_seg; s += kConsumers) {
             if (s >= g.seg_lo && s < g.seg_hi) {
@@ -482,63 +524,71 @@ __global__ void __launch_bounds__(kTmaThreads, kCtasPerSm) rows_tma_kernel(const
           }
         }
         if (tid == 0) { a.row_loss[r] = 0.f; a.row_flags[r] = 0u; }
-        __syncwarp();
-        if (lane == 0) mbar_arrive(&ctrl->own_empty[b]);
         continue;
       }
+      const uint32_t own_parity = (uint32_t)v & 1u;
 
-      // ---------------- pass over the resident own row: max, then sum exp / sum z
-      // Interior segments take the packed path; the (at most two) ragged edge segments are handled
-      // element by element by one thread each.
-      const int e0 = g.seg_lo > 0 ? 0 : -1;
-      const int e1 = (g.seg_hi < g.n_seg && !(e0 == 0 && g.n_seg == 1)) ? g.n_seg - 1 : -1;
-      const int my_edge = (tid == 0) ? e0 : (tid == 32 ? e1 : -1);
+      // ---------------- first pass over the own row, piece by piece as it lands: the maximum
       typename SegOps<T>::macc mx = SegOps<T>::neg_inf();
-      for (int s = g.seg_lo + tid; s < g.seg_hi; s += kConsumers)
-        mx = SegOps<T>::mmax(mx, SegOps<T>::fold(*reinterpret_cast<const uint4*>(img + (size_t)s * 16)));
-      float m_t = SegOps<T>::to_float(mx);
-      if (my_edge >= 0) {
-        float z[V];
-        SegOps<T>::unpack(*reinterpret_cast<const uint4*>(img + (size_t)my_edge * 16), z);
+      float m_edge = -INFINITY;
+      for (int k = 0; k < n_pieces; ++k) {
+        wait_bounded(&ctrl->own_full[k], own_parity, ctrl, a.hdr);
 #pragma unroll
-        for (int i = 0; i < V; ++i) {
-          const int64_t c = (int64_t)my_edge * V - g.head + i;
-          if (c >= 0 && c < C) m_t = fmaxf(m_t, z[i]);
+        for (int u = 0; u < kSegPerThread; ++u) {
+          const int s = k * kSegPerChunk + u * kConsumers + tid;
+          if (s >= g.seg_lo && s < g.seg_hi) {
+            mx = SegOps<T>::mmax(mx, SegOps<T>::fold(*reinterpret_cast<const uint4*>(img + (size_t)s * 16)));
+          } else if (s < g.n_seg) {
+            float z[V];
+            SegOps<T>::unpack(*reinterpret_cast<const uint4*>(img + (size_t)s * 16), z);
+#pragma unroll
+            for (int i = 0; i < V; ++i) {
+              const int64_t c = (int64_t)s * V - g.head + i;
+              if (c >= 0 && c < C) m_edge = fmaxf(m_edge, z[i]);
+            }
+          }
         }
       }
+      const float m_t = fmaxf(SegOps<T>::to_float(mx), m_edge);
       float mm[1] = {m_t};
       red.max(mm);
       const float m = mm[0];
+
+      // ---------------- second sweep: sum exp(z - m), sum z
       const float2 l2e2 = make_float2(kLog2e, kLog2e);
       const float2 nml2 = make_float2(-m * kLog2e, -m * kLog2e);
       float2 s2[H], zs2[H];
 #pragma unroll
       for (int i = 0; i < H; ++i) { s2[i] = make_float2(0.f, 0.f); zs2[i] = make_float2(0.f, 0.f); }
-      for (int s = g.seg_lo + tid; s < g.seg_hi; s += kConsumers) {
-        float2 z2[H];
-        SegOps<T>::unpack2(*reinterpret_cast<const uint4*>(img + (size_t)s * 16), z2);
-#pragma unroll
-        for (int i = 0; i < H; ++i) {
-          s2[i] = __fadd2_rn(s2[i], exp_shift2<T>(z2[i], m, l2e2, nml2));
-          zs2[i] = __fadd2_rn(zs2[i], z2[i]);
-        }
-      }
       float acc[2] = {0.f, 0.f};
+      for (int k = 0; k < n_pieces; ++k) {
 #pragma unroll
-      for (int i = 0; i < H; ++i) { acc[0] += s2[i].x + s2[i].y; acc[1] += zs2[i].x + zs2[i].y; }
-      if (my_edge >= 0) {
-        float z[V];
-        SegOps<T>::unpack(*reinterpret_cast<const uint4*>(img + (size_t)my_edge * 16), z);
+        for (int u = 0; u < kSegPerThread; ++u) {
+          const int s = k * kSegPerChunk + u * kConsumers + tid;
+          if (s >= g.seg_lo && s < g.seg_hi) {
+            float2 z2[H];
+            SegOps<T>::unpack2(*reinterpret_cast<const uint4*>(img + (size_t)s * 16), z2);
 #pragma unroll
-        for (int i = 0; i < V; ++i) {
-          const int64_t c = (int64_t)my_edge * V - g.head + i;
-          if (c >= 0 && c < C) {
-            const float2 e = exp_shift2<T>(make_float2(z[i], z[i]), m, l2e2, nml2);
-            acc[0] += e.x;
-            acc[1] += z[i];
+            for (int i = 0; i < H; ++i) {
+              s2[i] = __fadd2_rn(s2[i], exp_shift2<T>(z2[i], m, l2e2, nml2));
+              zs2[i] = __fadd2_rn(zs2[i], z2[i]);
+            }
+          } else if (s < g.n_seg) {
+            float z[V];
+            SegOps<T>::unpack(*reinterpret_cast<const uint4*>(img + (size_t)s * 16), z);
+#pragma unroll
+            for (int i = 0; i < V; ++i) {
+              const int64_t c = (int64_t)s * V - g.head + i;
+              if (c >= 0 && c < C) {
+                acc[0] += exp_shift2<T>(make_float2(z[i], z[i]), m, l2e2, nml2).x;
+                acc[1] += z[i];
+              }
+            }
           }
         }
       }
+#pragma unroll
+      for (int i = 0; i < H; ++i) { acc[0] += s2[i].x + s2[i].y; acc[1] += zs2[i].x + zs2[i].y; }
       red.sum(acc);
       const float S = acc[0], sum_z = acc[1];
       const float zy = Elem<T>::to_f32(reinterpret_cast<const T*>(img)[g.head + y]);
@@ -549,16 +599,19 @@ __global__ void __launch_bounds__(kTmaThreads, kCtasPerSm) rows_tma_kernel(const
       if (a.want_flags) {
         int first = 0x7fffffff;
         if (m_t == m) {
-          if (my_edge == e0 && e0 >= 0) first = first_equal<T>(img, e0, g.head, C, m);
-          for (int s = g.seg_lo + tid; s < g.seg_hi && first == 0x7fffffff; s += kConsumers)
-            first = first_equal<T>(img, s, g.head, C, m);
-          if (first == 0x7fffffff && my_edge == e1 && e1 >= 0) first = first_equal<T>(img, e1, g.head, C, m);
+          for (int k = 0; k < n_pieces && first == 0x7fffffff; ++k) {
+#pragma unroll
+            for (int u = 0; u < kSegPerThread; ++u) {
+              const int s = k * kSegPerChunk + u * kConsumers + tid;
+              if (s < g.n_seg && first == 0x7fffffff) first = first_equal<T>(img, s, g.head, C, m);
+            }
+          }
         }
         a_own = red.min_int(first);
       }
       const int seg_a = a.want_flags ? (g.head + a_own) / V : -1;
 
-      // ---------------- stream the peers chunk by chunk, write the gradient
+      // ---------------- stream the peers chunk by chunk, write the gradient, release the own pieces
       const float cp = w / S;                                                     // e_c -> w * p_c
       const float cd = with_term ? w * a.alpha * (2.f / (float)C) * inv_P : 0.f;  // sum_j d -> w * alpha * dD
       const float cq = w * a.eps / (float)C;
@@ -572,8 +625,7 @@ __global__ void __launch_bounds__(kTmaThreads, kCtasPerSm) rows_tma_kernel(const
 #pragma unroll
       for (int j = 0; j < PD; ++j) { lt[j] = SegOps<T>::neg_inf(); ge[j] = SegOps<T>::neg_inf(); za[j] = -INFINITY; }
 
-      const int n_chunks = (g.n_seg + kSegPerChunk - 1) / kSegPerChunk;
-      for (int k = 0; k < n_chunks; ++k) {
+      for (int k = 0; k < n_pieces; ++k) {
         float2 z2[kSegPerThread][H], sd2[kSegPerThread][H];
         bool active[kSegPerThread], special[kSegPerThread], edge[kSegPerThread];
         int seg[kSegPerThread];
@@ -661,7 +713,11 @@ __global__ void __launch_bounds__(kTmaThreads, kCtasPerSm) rows_tma_kernel(const
             }
           }
         }
+        // this piece of the own row is no longer needed: the producer may refill it
+        __syncwarp();
+        if (lane == 0) mbar_arrive(&ctrl->own_empty[k]);
       }
+      ++v;
 
       // ---------------- row results
       float dsum[1] = {dist2.x + dist2.y};
@@ -689,8 +745,6 @@ __global__ void __launch_bounds__(kTmaThreads, kCtasPerSm) rows_tma_kernel(const
         a.row_loss[r] = with_term ? fmaf(a.alpha, D, ce) : ce;
         a.row_flags[r] = flags;
       }
-      __syncwarp();
-      if (lane == 0) mbar_arrive(&ctrl->own_empty[b]);
     }
   }
 
@@ -719,25 +773,32 @@ static bool tma_config(const KArgs& a, int dtype, int smem_optin, TmaCfg* out) {
   uintptr_t bits = reinterpret_cast<uintptr_t>(a.own) | reinterpret_cast<uintptr_t>(a.grad);
   for (int j = 0; j < a.n_peers; ++j) bits |= reinterpret_cast<uintptr_t>(a.peers[j]);
   if (bits & 15u) return false;
-  const int64_t own_buf = ((row_bytes + 32 + 127) / 128) * 128;
-  // per-CTA share of the SM's shared memory (1 KiB per CTA is reserved by the system)
-  const int64_t avail = (kCtasPerSm == 1 ? (int64_t)smem_optin : ((int64_t)smem_optin + 1024) / kCtasPerSm - 1024) - kCtrlBytes;
-  TmaCfg c;
-  c.own_buf_bytes = (uint32_t)own_buf;
-  const int min_stages = a.n_peers > 0 ? 3 : 1;
-  if (2 * own_buf + (int64_t)(a.n_peers > 0 ? 4 : 1) * kChunkBytes <= avail) {
-    c.own_bufs = 2;
-  } else if (own_buf + (int64_t)min_stages * kChunkBytes <= avail) {
-    c.own_bufs = 1;
-  } else {
-    return false;
+  const int64_t n_seg_max = dtype == CODISTILL_F32 ? max_row_segments<float>(a.row_stride, a.classes)
+                                                   : max_row_segments<__nv_bfloat16>(a.row_stride, a.classes);
+  // Two CTAs of 8 consumer warps per SM when the row buffer leaves room for a ring in half an SM's
+  // shared memory, otherwise one CTA of 16 consumer warps.
+  for (int pass = 0; pass < 2; ++pass) {
+    TmaCfg c;
+    c.consumer_warps = pass == 0 ? 8 : 16;
+    c.ctas_per_sm = pass == 0 ? 2 : 1;
+    c.chunk_bytes = (uint32_t)c.consumer_warps * 32u * kSegPerThread * 16u;
+    const int64_t seg_per_chunk = c.chunk_bytes / 16;
+    c.pieces = (int)((n_seg_max + seg_per_chunk - 1) / seg_per_chunk);
+    if (c.pieces > kMaxPieces) continue;
+    const int64_t own_buf = (int64_t)c.pieces * c.chunk_bytes;  // whole pieces, so that every piece has a home
+    const int64_t per_cta = c.ctas_per_sm == 1 ? (int64_t)smem_optin : ((int64_t)smem_optin + 1024) / c.ctas_per_sm - 1024;
+    int64_t st = (per_cta - kCtrlBytes - own_buf) / c.chunk_bytes;
+    const int min_stages = a.n_peers > 0 ? (pass == 0 ? 4 : 2) : 0;
+    if (st < min_stages) continue;
+    if (st > kMaxStages) st = kMaxStages;
+    if (a.n_peers == 0) st = 1;
+    c.stages = (int)st;
+    c.own_buf_bytes = (uint32_t)own_buf;
+    c.smem_bytes = (uint32_t)(kCtrlBytes + own_buf + st * c.chunk_bytes);
+    *out = c;
+    return true;
   }
-  int64_t st = (avail - (int64_t)c.own_bufs * own_buf) / kChunkBytes;
-  if (st > kMaxStages) st = kMaxStages;
-  c.stages = (int)st;
-  c.smem_bytes = (uint32_t)(kCtrlBytes + (int64_t)c.own_bufs * own_buf + (int64_t)c.stages * kChunkBytes);
-  *out = c;
-  return true;
+  return false;
 }
 
 bool tma_supported(const KArgs& a, int dtype, int smem_optin) {
@@ -745,27 +806,30 @@ bool tma_supported(const KArgs& a, int dtype, int smem_optin) {
   return tma_config(a, dtype, smem_optin, &c);
 }
 
-template <typename T, int P, bool PW>
+template <typename T, int P, bool PW, int NCW>
 static cudaError_t launch_one(const KArgs& a, const TmaCfg& c, int grid, cudaStream_t stream) {
-  cudaError_t e = cudaFuncSetAttribute(rows_tma_kernel<T, P, PW>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)c.smem_bytes);
+  cudaError_t e = cudaFuncSetAttribute(rows_tma_kernel<T, P, PW, NCW>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)c.smem_bytes);
   if (e != cudaSuccess) return e;
-  rows_tma_kernel<T, P, PW><<<grid, kTmaThreads, c.smem_bytes, stream>>>(a, c);
+  rows_tma_kernel<T, P, PW, NCW><<<grid, NCW * 32 + kProducerThreads, c.smem_bytes, stream>>>(a, c);
   return cudaGetLastError();
 }
 
-// PW: the loss sums squared pairwise differences (Algorithm 1); otherwise the squared difference to
-// the averaged peer.  With one peer the two coincide.
-template <typename T>
-static cudaError_t launch_dtype(const KArgs& a, const TmaCfg& c, int grid, cudaStream_t stream) {
-  const bool pw = a.peer_reduce == CODISTILL_PEERS_PAIRWISE_MEAN;
+template <typename T, int NCW>
+static cudaError_t launch_peers(const KArgs& a, const TmaCfg& c, int grid, cudaStream_t stream) {
+  const bool pw = a.peer_reduce == CODISTILL_PEERS_PAIRWISE_MEAN;  // with one peer both readings coincide
   switch (a.n_peers) {
-    case 0: return launch_one<T, 0, true>(a, c, grid, stream);
-    case 1: return launch_one<T, 1, true>(a, c, grid, stream);
-    case 2: return pw ? launch_one<T, 2, true>(a, c, grid, stream) : launch_one<T, 2, false>(a, c, grid, stream);
-    case 3: return pw ? launch_one<T, 3, true>(a, c, grid, stream) : launch_one<T, 3, false>(a, c, grid, stream);
-    case 7: return pw ? launch_one<T, 7, true>(a, c, grid, stream) : launch_one<T, 7, false>(a, c, grid, stream);
+    case 0: return launch_one<T, 0, true, NCW>(a, c, grid, stream);
+    case 1: return launch_one<T, 1, true, NCW>(a, c, grid, stream);
+    case 2: return pw ? launch_one<T, 2, true, NCW>(a, c, grid, stream) : launch_one<T, 2, false, NCW>(a, c, grid, stream);
+    case 3: return pw ? launch_one<T, 3, true, NCW>(a, c, grid, stream) : launch_one<T, 3, false, NCW>(a, c, grid, stream);
+    case 7: return pw ? launch_one<T, 7, true, NCW>(a, c, grid, stream) : launch_one<T, 7, false, NCW>(a, c, grid, stream);
     default: return cudaErrorNotSupported;
   }
+}
+
+template <typename T>
+static cudaError_t launch_dtype(const KArgs& a, const TmaCfg& c, int grid, cudaStream_t stream) {
+  return c.consumer_warps == 8 ? launch_peers<T, 8>(a, c, grid, stream) : launch_peers<T, 16>(a, c, grid, stream);
 }
 
 cudaError_t launch_tma(const KArgs& a, int dtype, int num_sms, int smem_optin, cudaStream_t stream) {
@@ -773,7 +837,7 @@ cudaError_t launch_tma(const KArgs& a, int dtype, int num_sms, int smem_optin, c
   if (!tma_config(a, dtype, smem_optin, &c)) return cudaErrorNotSupported;
   const int64_t rows = a.row_end - a.row_begin;
   if (rows <= 0) return cudaSuccess;
-  const int64_t slots = (int64_t)num_sms * kCtasPerSm;
+  const int64_t slots = (int64_t)num_sms * c.ctas_per_sm;
   const int grid = (int)(rows < slots ? rows : slots);
   return dtype == CODISTILL_F32 ? launch_dtype<float>(a, c, grid, stream) : launch_dtype<__nv_bfloat16>(a, c, grid, stream);
 }
