@@ -60,7 +60,8 @@ struct Ctrl {  // lives at the start of dynamic shared memory
   RowInfo info[kInfoSlots];
   int abort_flag;
   int last_flag;
-  float red[2][kMaxConsumerWarps * 24];  // reduction scratch of the consumers, two alternating halves
+  float red[2][kMaxConsumerWarps * 4];   // reduction scratch of the consumers, two alternating halves
+  float endred[kMaxConsumerWarps * 24];  // per-warp partials of the end-of-row reduction (read by consumer warp 0)
   double fin[32];
 };
 static_assert(sizeof(Ctrl) <= kCtrlBytes, "control block fits its slot");
@@ -260,6 +261,17 @@ struct ConsumerReduce {
     for (int k = 0; k < N; ++k) v[k] = warp_max(lane < NCW ? s[k * NCW + lane] : -INFINITY);
     toggle ^= 1;
   }
+  // larger value wins; on equal values the smaller index wins
+  __device__ __forceinline__ void argmax(float& v, int& i) {
+    float* s = ctrl->red[toggle];
+    warp_argmax(v, i);
+    if (lane == 0) { s[warp] = v; reinterpret_cast<int*>(s)[NCW + warp] = i; }
+    bar();
+    v = lane < NCW ? s[lane] : -INFINITY;
+    i = lane < NCW ? reinterpret_cast<int*>(s)[NCW + lane] : 0x7fffffff;
+    warp_argmax(v, i);
+    toggle ^= 1;
+  }
   __device__ __forceinline__ int min_int(int v) {
     int* s = reinterpret_cast<int*>(ctrl->red[toggle]);
 #pragma unroll
@@ -455,7 +467,9 @@ rows_tma_kernel(const __grid_constant__ KArgs a, const TmaCfg cfg) {
       for (int k = 0; k < n_pieces; ++k) wait_bounded(&ctrl->own_full[k], (v - 1) & 1, ctrl, a.hdr);
   } else if (warp == 1) {
     // ============================== peer producer ==============================
-    uint32_t q = 0;  // ring items issued so far
+    uint32_t q = 0;          // ring items issued so far
+    int st = 0;              // stage of the next item
+    uint32_t st_phase = 0;   // phase bit of that stage's next use
     for (int it = 0;; ++it) {
       const int slot = it % kInfoSlots;
       wait_bounded(&ctrl->info_full[slot], (it / kInfoSlots) & 1, ctrl, a.hdr);
@@ -472,10 +486,10 @@ rows_tma_kernel(const __grid_constant__ KArgs a, const TmaCfg cfg) {
         if (end < begin) end = begin;
 #pragma unroll 1
         for (int j = 0; j < P; ++j, ++q) {
-          const int s = q % n_stage;
-          if (q >= (uint32_t)n_stage) wait_bounded(&ctrl->ring_empty[s], ((q / n_stage) - 1) & 1, ctrl, a.hdr);
-          produce_copy<T>(ring_base + (size_t)s * kChunkBytes, reinterpret_cast<const char*>(a.peers[j]) + rc.row_off, begin, end,
-                          rc.tma_limit, rc.valid_end, &ctrl->ring_full[s], lane);
+          if (q >= (uint32_t)n_stage) wait_bounded(&ctrl->ring_empty[st], st_phase ^ 1u, ctrl, a.hdr);
+          produce_copy<T>(ring_base + (size_t)st * kChunkBytes, reinterpret_cast<const char*>(a.peers[j]) + rc.row_off, begin, end,
+                          rc.tma_limit, rc.valid_end, &ctrl->ring_full[st], lane);
+          if (++st == n_stage) { st = 0; st_phase ^= 1u; }
         }
       }
     }
@@ -493,8 +507,9 @@ rows_tma_kernel(const __grid_constant__ KArgs a, const TmaCfg cfg) {
       w = 1.f / (float)(nv > 1 ? nv : 1);
     }
     const float inv_P = P >= 1 ? 1.f / (float)P : 0.f;
-    uint32_t q = 0;
-    int v = 0;  // valid rows processed so far
+    int st = 0;              // ring stage of the next item
+    uint32_t st_phase = 0;   // its phase bit
+    int v = 0;               // valid rows processed so far
     for (int it = 0;; ++it) {
       const int slot = it % kInfoSlots;
       wait_bounded(&ctrl->info_full[slot], (it / kInfoSlots) & 1, ctrl, a.hdr);
@@ -528,31 +543,37 @@ rows_tma_kernel(const __grid_constant__ KArgs a, const TmaCfg cfg) {
       }
       const uint32_t own_parity = (uint32_t)v & 1u;
 
-      // ---------------- first pass over the own row, piece by piece as it lands: the maximum
-      typename SegOps<T>::macc mx = SegOps<T>::neg_inf();
-      float m_edge = -INFINITY;
+      // ---------------- first pass over the own row, piece by piece as it lands: maximum and the
+      // first segment that holds it (a thread visits its segments in rising order, so a strict
+      // comparison keeps the first)
+      float best = -INFINITY;
+      int best_seg = 0x7fffffff;
       for (int k = 0; k < n_pieces; ++k) {
         wait_bounded(&ctrl->own_full[k], own_parity, ctrl, a.hdr);
 #pragma unroll
         for (int u = 0; u < kSegPerThread; ++u) {
           const int s = k * kSegPerChunk + u * kConsumers + tid;
+          float fm = -INFINITY;
           if (s >= g.seg_lo && s < g.seg_hi) {
-            mx = SegOps<T>::mmax(mx, SegOps<T>::fold(*reinterpret_cast<const uint4*>(img + (size_t)s * 16)));
+            fm = SegOps<T>::to_float(SegOps<T>::fold(*reinterpret_cast<const uint4*>(img + (size_t)s * 16)));
           } else if (s < g.n_seg) {
             float z[V];
             SegOps<T>::unpack(*reinterpret_cast<const uint4*>(img + (size_t)s * 16), z);
 #pragma unroll
             for (int i = 0; i < V; ++i) {
               const int64_t c = (int64_t)s * V - g.head + i;
-              if (c >= 0 && c < C) m_edge = fmaxf(m_edge, z[i]);
+              if (c >= 0 && c < C) fm = fmaxf(fm, z[i]);
             }
           }
+          if (fm > best) { best = fm; best_seg = s; }
         }
       }
-      const float m_t = fmaxf(SegOps<T>::to_float(mx), m_edge);
-      float mm[1] = {m_t};
-      red.max(mm);
-      const float m = mm[0];
+      red.argmax(best, best_seg);
+      if (best_seg >= g.n_seg) best_seg = 0;  // NaN rows: keep the read below inside the row image
+      const float m = best;
+      // every thread reads the winning segment: first column that attains the maximum
+      const int a_own = first_equal<T>(img, best_seg, g.head, C, m);
+      const int seg_a = a.want_flags ? best_seg : -1;
 
       // ---------------- second sweep: sum exp(z - m), sum z
       const float2 l2e2 = make_float2(kLog2e, kLog2e);
@@ -594,23 +615,6 @@ rows_tma_kernel(const __grid_constant__ KArgs a, const TmaCfg cfg) {
       const float zy = Elem<T>::to_f32(reinterpret_cast<const T*>(img)[g.head + y]);
       const float ce = (m + logf(S)) - (1.f - a.eps) * zy - (a.eps / (float)C) * sum_z;
 
-      // ---------------- first arg-max of the own row (only threads that hold the maximum rescan)
-      int a_own = 0;
-      if (a.want_flags) {
-        int first = 0x7fffffff;
-        if (m_t == m) {
-          for (int k = 0; k < n_pieces && first == 0x7fffffff; ++k) {
-#pragma unroll
-            for (int u = 0; u < kSegPerThread; ++u) {
-              const int s = k * kSegPerChunk + u * kConsumers + tid;
-              if (s < g.n_seg && first == 0x7fffffff) first = first_equal<T>(img, s, g.head, C, m);
-            }
-          }
-        }
-        a_own = red.min_int(first);
-      }
-      const int seg_a = a.want_flags ? (g.head + a_own) / V : -1;
-
       // ---------------- stream the peers chunk by chunk, write the gradient, release the own pieces
       const float cp = w / S;                                                     // e_c -> w * p_c
       const float cd = with_term ? w * a.alpha * (2.f / (float)C) * inv_P : 0.f;  // sum_j d -> w * alpha * dD
@@ -639,12 +643,37 @@ rows_tma_kernel(const __grid_constant__ KArgs a, const TmaCfg cfg) {
           for (int i = 0; i < H; ++i) { z2[u][i] = make_float2(0.f, 0.f); sd2[u][i] = make_float2(0.f, 0.f); }
           if (active[u]) SegOps<T>::unpack2(*reinterpret_cast<const uint4*>(img + (size_t)seg[u] * 16), z2[u]);
         }
+        bool all_fast = with_term;
+#pragma unroll
+        for (int u = 0; u < kSegPerThread; ++u) all_fast = all_fast && active[u] && !special[u];
         if (stream_peers) {
 #pragma unroll
-          for (int j = 0; j < P; ++j, ++q) {
-            const int st = q % n_stage;
-            wait_bounded(&ctrl->ring_full[st], (q / n_stage) & 1, ctrl, a.hdr);
+          for (int j = 0; j < P; ++j) {
+            wait_bounded(&ctrl->ring_full[st], st_phase, ctrl, a.hdr);
             const char* chunk = ring_base + (size_t)st * kChunkBytes;
+            if (all_fast) {  // both segments lie wholly inside the row and away from the arg-max column
+              uint4 raw[kSegPerThread];
+#pragma unroll
+              for (int u = 0; u < kSegPerThread; ++u)
+                raw[u] = *reinterpret_cast<const uint4*>(chunk + (size_t)(u * kConsumers + tid) * 16);
+#pragma unroll
+              for (int u = 0; u < kSegPerThread; ++u) {
+                float2 v2[H];
+                SegOps<T>::unpack2(raw[u], v2);
+#pragma unroll
+                for (int i = 0; i < H; ++i) {
+                  const float2 d = __ffma2_rn(v2[i], neg1, z2[u][i]);
+                  if constexpr (P == 1) sd2[u][i] = d; else sd2[u][i] = __fadd2_rn(sd2[u][i], d);
+                  if constexpr (PW) dist2 = __ffma2_rn(d, d, dist2);
+                }
+                if (a.want_flags) {
+                  const typename SegOps<T>::macc f = SegOps<T>::fold(raw[u]);
+                  const bool before = seg[u] < seg_a;
+                  lt[j] = before ? SegOps<T>::mmax(lt[j], f) : lt[j];
+                  ge[j] = before ? ge[j] : SegOps<T>::mmax(ge[j], f);
+                }
+              }
+            } else
 #pragma unroll
             for (int u = 0; u < kSegPerThread; ++u) {
               if (!active[u]) continue;
@@ -680,6 +709,7 @@ rows_tma_kernel(const __grid_constant__ KArgs a, const TmaCfg cfg) {
             }
             __syncwarp();
             if (lane == 0) mbar_arrive(&ctrl->ring_empty[st]);
+            if (++st == n_stage) { st = 0; st_phase ^= 1u; }
           }
         }
         // gradient of this chunk's segments
@@ -719,31 +749,45 @@ rows_tma_kernel(const __grid_constant__ KArgs a, const TmaCfg cfg) {
       }
       ++v;
 
-      // ---------------- row results
-      float dsum[1] = {dist2.x + dist2.y};
-      if (with_term) red.sum(dsum);
-      uint32_t flags = 0u;
-      if (a.want_flags) {
-        flags = (a_own == y) ? 1u : 0u;
-        if (P >= 1) {
-          float mxv[3 * PD];
+      // ---------------- row results: one merged reduction that only consumer warp 0 waits for
+      {
+        float part[1 + 3 * PD];
+        part[0] = warp_sum(dist2.x + dist2.y);
 #pragma unroll
-          for (int j = 0; j < PD; ++j) {
-            mxv[3 * j] = SegOps<T>::to_float(lt[j]);
-            mxv[3 * j + 1] = SegOps<T>::to_float(ge[j]);
-            mxv[3 * j + 2] = za[j];
-          }
-          red.max(mxv);
-#pragma unroll
-          for (int j = 0; j < PD; ++j)
-            if (mxv[3 * j + 2] >= mxv[3 * j + 1] && mxv[3 * j] < mxv[3 * j + 2]) flags |= (2u << j);
+        for (int j = 0; j < PD; ++j) {
+          part[1 + 3 * j] = warp_max(SegOps<T>::to_float(lt[j]));
+          part[2 + 3 * j] = warp_max(SegOps<T>::to_float(ge[j]));
+          part[3 + 3 * j] = warp_max(za[j]);
         }
-      }
-      if (tid == 0) {
-        float D = 0.f;
-        if (with_term) D = PW ? dsum[0] * inv_P / (float)C : dsum[0] * inv_P * inv_P / (float)C;
-        a.row_loss[r] = with_term ? fmaf(a.alpha, D, ce) : ce;
-        a.row_flags[r] = flags;
+        const int cw = warp - 2;
+        if (lane == 0) {
+#pragma unroll
+          for (int i = 0; i < 1 + 3 * PD; ++i) ctrl->endred[i * NCW + cw] = part[i];
+        }
+        __threadfence_block();
+        if (cw != 0) {
+          asm volatile("bar.arrive 2, %0;" ::"n"(NCW * 32) : "memory");
+        } else {
+          asm volatile("bar.sync 2, %0;" ::"n"(NCW * 32) : "memory");
+          float dsum = warp_sum(lane < NCW ? ctrl->endred[lane] : 0.f);
+          uint32_t flags = 0u;
+          if (a.want_flags) {
+            flags = (a_own == y) ? 1u : 0u;
+#pragma unroll
+            for (int j = 0; j < P; ++j) {
+              const float ltv = warp_max(lane < NCW ? ctrl->endred[(1 + 3 * j) * NCW + lane] : -INFINITY);
+              const float gev = warp_max(lane < NCW ? ctrl->endred[(2 + 3 * j) * NCW + lane] : -INFINITY);
+              const float zav = warp_max(lane < NCW ? ctrl->endred[(3 + 3 * j) * NCW + lane] : -INFINITY);
+              if (zav >= gev && ltv < zav) flags |= (2u << j);
+            }
+          }
+          if (lane == 0) {
+            float D = 0.f;
+            if (with_term) D = PW ? dsum * inv_P / (float)C : dsum * inv_P * inv_P / (float)C;
+            a.row_loss[r] = with_term ? fmaf(a.alpha, D, ce) : ce;
+            a.row_flags[r] = flags;
+          }
+        }
       }
     }
   }
