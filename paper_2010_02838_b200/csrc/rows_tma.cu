@@ -10,10 +10,13 @@
 //           row streams in behind the current row's second pass.
 //   warp 1  peer producer: streams the n-1 peer rows chunk by chunk (chunk-major: chunk k of peer
 //           0, 1, ..., then chunk k+1) through the ring of stages.
-//   others  consumers: first pass over the resident own row (max, sum exp, sum z, first arg-max),
-//           then per chunk: consume the peers from the ring (sum_j (z - z_j), sum_j (z - z_j)^2,
-//           what the arg-max agreement needs), write the gradient with 128-bit stores, release the
-//           own piece.
+//   warp 2  service warp: writes the all-zero gradient rows of masked rows and turns the consumers'
+//           per-warp partial results of a finished row into the per-row loss and flag word, off
+//           the consumers' critical path.
+//   others  consumers: one sweep over the resident own row as its pieces land (online softmax:
+//           running max, sum exp, sum z, first arg-max), one block reduction, then per chunk:
+//           consume the peers from the ring (sum_j (z - z_j), sum_j (z - z_j)^2, what the arg-max
+//           agreement needs), write the gradient with 128-bit stores, release the own piece.
 // Every logit is read from HBM exactly once and the gradient is written once.
 //
 // A "row image" is the 16-byte aligned byte range that contains the row: rows whose byte length
@@ -27,8 +30,8 @@ namespace codistill {
 constexpr int kMaxStages = 12;
 constexpr int kMaxPieces = 32;
 constexpr int kInfoSlots = 4;
-constexpr int kCtrlBytes = 5120;
-constexpr int kProducerThreads = 64;   // warp 0: scheduler + own row, warp 1: peers
+constexpr int kCtrlBytes = 6144;
+constexpr int kProducerThreads = 64;   // warp 0: scheduler + own row, warp 1: peers + service
 constexpr int kSegPerThread = 2;       // 16-byte segments per consumer thread per chunk
 constexpr int kMaxConsumerWarps = 16;
 constexpr uint32_t kBulkPieceBytes = 32768;
@@ -60,8 +63,12 @@ struct Ctrl {  // lives at the start of dynamic shared memory
   RowInfo info[kInfoSlots];
   int abort_flag;
   int last_flag;
-  float red[2][kMaxConsumerWarps * 4];   // reduction scratch of the consumers, two alternating halves
-  float endred[kMaxConsumerWarps * 24];  // per-warp partials of the end-of-row reduction (read by consumer warp 0)
+  uint64_t end_full[2];    // consumers -> service warp: partial results of a row are in endred[par]
+  uint64_t end_empty[2];   // service warp -> consumers: endred[par] may be overwritten
+  float red[2][kMaxConsumerWarps * 4];      // reduction scratch of the consumers, two alternating halves
+  float endred[2][kMaxConsumerWarps * 24];  // per-warp partials of the end-of-row reduction
+  float end_ce[2];                          // task loss of the row
+  int end_correct[2];                       // arg-max == label
   double fin[32];
 };
 static_assert(sizeof(Ctrl) <= kCtrlBytes, "control block fits its slot");
@@ -199,6 +206,13 @@ __device__ __forceinline__ float2 exp_shift2(float2 z, float m, float2 l2e, floa
     const float2 t = __ffma2_rn(z, l2e, neg_m_l2e);
     return make_float2(ex2_approx(t.x), ex2_approx(t.y));
   }
+}
+
+// 2^x for the rescaling factors of the online softmax: exact enough for the 1e-6 gradient tolerance of
+// fp32 logits, the bare hardware instruction for bf16 logits.
+template <typename T>
+__device__ __forceinline__ float rescale_exp2(float x) {
+  if constexpr (sizeof(T) == 4) return exp2f(x); else return ex2_approx(x);
 }
 
 // Geometry of one row image.
@@ -410,6 +424,7 @@ rows_tma_kernel(const __grid_constant__ KArgs a, const TmaCfg cfg) {
     for (int k = 0; k < kMaxPieces; ++k) { mbar_init(&ctrl->own_full[k], 1); mbar_init(&ctrl->own_empty[k], NCW); }
     for (int s = 0; s < kMaxStages; ++s) { mbar_init(&ctrl->ring_full[s], 1); mbar_init(&ctrl->ring_empty[s], NCW); }
     for (int s = 0; s < kInfoSlots; ++s) { mbar_init(&ctrl->info_full[s], 1); mbar_init(&ctrl->info_empty[s], NCW + 1); }
+    for (int s = 0; s < 2; ++s) { mbar_init(&ctrl->end_full[s], NCW); mbar_init(&ctrl->end_empty[s], 1); }
     ctrl->abort_flag = 0;
     ctrl->last_flag = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -466,10 +481,40 @@ rows_tma_kernel(const __grid_constant__ KArgs a, const TmaCfg cfg) {
     if (v >= 1)
       for (int k = 0; k < n_pieces; ++k) wait_bounded(&ctrl->own_full[k], (v - 1) & 1, ctrl, a.hdr);
   } else if (warp == 1) {
-    // ============================== peer producer ==============================
+    // ============================== peer producer + service ==============================
+    const float inv_P = P >= 1 ? 1.f / (float)P : 0.f;
+    // Turns the consumers' per-warp partials of valid row number `vv` into its loss and flag word.
+    auto finish_row = [&](int vv, long long row) {
+      const int par = vv & 1;
+      wait_bounded(&ctrl->end_full[par], (uint32_t)(vv >> 1) & 1u, ctrl, a.hdr);
+      const float* er = ctrl->endred[par];
+      const float dsum = warp_sum(lane < NCW ? er[lane] : 0.f);
+      uint32_t flags = 0u;
+      if (a.want_flags) {
+        flags = ctrl->end_correct[par] ? 1u : 0u;
+#pragma unroll
+        for (int j = 0; j < P; ++j) {
+          const float ltv = warp_max(lane < NCW ? er[(1 + 3 * j) * NCW + lane] : -INFINITY);
+          const float gev = warp_max(lane < NCW ? er[(2 + 3 * j) * NCW + lane] : -INFINITY);
+          const float zav = warp_max(lane < NCW ? er[(3 + 3 * j) * NCW + lane] : -INFINITY);
+          if (zav >= gev && ltv < zav) flags |= (2u << j);
+        }
+      }
+      const float ce = ctrl->end_ce[par];
+      __syncwarp();
+      if (lane == 0) {
+        mbar_arrive(&ctrl->end_empty[par]);
+        float D = 0.f;
+        if (with_term) D = PW ? dsum * inv_P / (float)C : dsum * inv_P * inv_P / (float)C;
+        a.row_loss[row] = with_term ? fmaf(a.alpha, D, ce) : ce;
+        a.row_flags[row] = flags;
+      }
+    };
     uint32_t q = 0;          // ring items issued so far
     int st = 0;              // stage of the next item
     uint32_t st_phase = 0;   // phase bit of that stage's next use
+    int v = 0;               // valid rows seen so far
+    long long prev_row[2] = {-1, -1};  // rows whose results are still to be finished (valid rows v-2, v-1)
     for (int it = 0;; ++it) {
       const int slot = it % kInfoSlots;
       wait_bounded(&ctrl->info_full[slot], (it / kInfoSlots) & 1, ctrl, a.hdr);
@@ -478,7 +523,32 @@ rows_tma_kernel(const __grid_constant__ KArgs a, const TmaCfg cfg) {
       __syncwarp();
       if (lane == 0) mbar_arrive(&ctrl->info_empty[slot]);
       if (r < 0) break;
-      if (!valid || !stream_peers) continue;
+      if (!valid) {  // masked row: zero gradient, no loss, no counts; nothing is copied for it
+        if (a.grad) {
+          const int64_t lr = r - a.row_begin;
+          const RowGeom g = row_geom<T>(lr, a.row_stride, C);
+          char* g_img = reinterpret_cast<char*>(a.grad) + lr * a.row_stride * ES - (int64_t)g.head * ES;
+          for (int s = lane; s < g.n_seg; s += 32) {
+            if (s >= g.seg_lo && s < g.seg_hi) {
+              *reinterpret_cast<uint4*>(g_img + (size_t)s * 16) = make_uint4(0u, 0u, 0u, 0u);
+            } else {
+#pragma unroll
+              for (int i = 0; i < V; ++i) {
+                const int64_t c = (int64_t)s * V - g.head + i;
+                if (c >= 0 && c < C) reinterpret_cast<T*>(g_img + (size_t)s * 16)[i] = Elem<T>::from_f32(0.f);
+              }
+            }
+          }
+        }
+        if (lane == 0) { a.row_loss[r] = 0.f; a.row_flags[r] = 0u; }
+        continue;
+      }
+      // The consumers are at most one row behind this warp, so valid row v-2 is complete: finish it
+      // before feeding row v (the consumers reuse its partial-result slot at the end of row v).
+      if (v >= 2) finish_row(v - 2, prev_row[v & 1]);
+      prev_row[v & 1] = r;
+      ++v;
+      if (!stream_peers) continue;
       const RowCopy rc = row_copy<T>(a, r);
       for (int k = 0; k < n_pieces; ++k) {
         const uint32_t begin = (uint32_t)k * kChunkBytes;
@@ -493,6 +563,9 @@ rows_tma_kernel(const __grid_constant__ KArgs a, const TmaCfg cfg) {
         }
       }
     }
+    // results of the last two valid rows
+    if (v >= 2) finish_row(v - 2, prev_row[v & 1]);
+    if (v >= 1) finish_row(v - 1, prev_row[(v - 1) & 1]);
     for (uint32_t i = 0; i < (uint32_t)n_stage && i < q; ++i) {
       const uint32_t qi = q - 1 - i;
       wait_bounded(&ctrl->ring_full[qi % n_stage], (qi / n_stage) & 1, ctrl, a.hdr);
@@ -524,41 +597,36 @@ rows_tma_kernel(const __grid_constant__ KArgs a, const TmaCfg cfg) {
       const char* img = own_buf;
       char* g_img = a.grad ? reinterpret_cast<char*>(a.grad) + lr * a.row_stride * ES - (int64_t)g.head * ES : nullptr;
 
-      if (!valid) {  // masked row: zero gradient, no loss, no counts; nothing was copied for it
-        if (g_img) {
-          for (int s = tid; s < g.n_seg; s += kConsumers) {
-            if (s >= g.seg_lo && s < g.seg_hi) {
-              *reinterpret_cast<uint4*>(g_img + (size_t)s * 16) = make_uint4(0u, 0u, 0u, 0u);
-            } else {
-#pragma unroll
-              for (int i = 0; i < V; ++i) {
-                const int64_t c = (int64_t)s * V - g.head + i;
-                if (c >= 0 && c < C) reinterpret_cast<T*>(g_img + (size_t)s * 16)[i] = Elem<T>::from_f32(0.f);
-              }
-            }
-          }
-        }
-        if (tid == 0) { a.row_loss[r] = 0.f; a.row_flags[r] = 0u; }
-        continue;
-      }
+      if (!valid) continue;  // masked rows are written by the service warp
       const uint32_t own_parity = (uint32_t)v & 1u;
 
-      // ---------------- first pass over the own row, piece by piece as it lands: maximum and the
-      // first segment that holds it (a thread visits its segments in rising order, so a strict
-      // comparison keeps the first)
-      float best = -INFINITY;
+      // ---------------- one sweep over the own row, piece by piece as it lands (online softmax):
+      // running maximum `best` with the first segment that attains it (a thread visits its segments
+      // in rising order, so a strict comparison keeps the first), sum exp(z - best), sum z.
+      const float2 l2e2 = make_float2(kLog2e, kLog2e);
+      float best = -3.0e38f;  // finite, so that the first rescale is exp2(-huge) = 0 and never NaN
       int best_seg = 0x7fffffff;
+      float2 s2[H], zs2[H];
+#pragma unroll
+      for (int i = 0; i < H; ++i) { s2[i] = make_float2(0.f, 0.f); zs2[i] = make_float2(0.f, 0.f); }
+      float s_edge = 0.f, z_edge = 0.f;  // contributions of ragged edge segments (relative to `best`)
       for (int k = 0; k < n_pieces; ++k) {
         wait_bounded(&ctrl->own_full[k], own_parity, ctrl, a.hdr);
+        uint4 raw[kSegPerThread];
+        bool inner[kSegPerThread], ragged[kSegPerThread];
+        const float old = best;
 #pragma unroll
         for (int u = 0; u < kSegPerThread; ++u) {
           const int s = k * kSegPerChunk + u * kConsumers + tid;
-          float fm = -INFINITY;
-          if (s >= g.seg_lo && s < g.seg_hi) {
-            fm = SegOps<T>::to_float(SegOps<T>::fold(*reinterpret_cast<const uint4*>(img + (size_t)s * 16)));
-          } else if (s < g.n_seg) {
+          inner[u] = s >= g.seg_lo && s < g.seg_hi;
+          ragged[u] = !inner[u] && s < g.n_seg;
+          float fm = -3.0e38f;
+          if (inner[u] || ragged[u]) raw[u] = *reinterpret_cast<const uint4*>(img + (size_t)s * 16);
+          if (inner[u]) {
+            fm = SegOps<T>::to_float(SegOps<T>::fold(raw[u]));
+          } else if (ragged[u]) {
             float z[V];
-            SegOps<T>::unpack(*reinterpret_cast<const uint4*>(img + (size_t)s * 16), z);
+            SegOps<T>::unpack(raw[u], z);
 #pragma unroll
             for (int i = 0; i < V; ++i) {
               const int64_t c = (int64_t)s * V - g.head + i;
@@ -567,51 +635,73 @@ rows_tma_kernel(const __grid_constant__ KArgs a, const TmaCfg cfg) {
           }
           if (fm > best) { best = fm; best_seg = s; }
         }
-      }
-      red.argmax(best, best_seg);
-      if (best_seg >= g.n_seg) best_seg = 0;  // NaN rows: keep the read below inside the row image
-      const float m = best;
-      // every thread reads the winning segment: first column that attains the maximum
-      const int a_own = first_equal<T>(img, best_seg, g.head, C, m);
-      const int seg_a = a.want_flags ? best_seg : -1;
-
-      // ---------------- second sweep: sum exp(z - m), sum z
-      const float2 l2e2 = make_float2(kLog2e, kLog2e);
-      const float2 nml2 = make_float2(-m * kLog2e, -m * kLog2e);
-      float2 s2[H], zs2[H];
+        // rescale what was summed so far to the new reference (factor 1 when it did not move)
+        const float scale = rescale_exp2<T>((old - best) * kLog2e);
+        const float2 scale2 = make_float2(scale, scale);
+        const float2 nml2k = make_float2(-best * kLog2e, -best * kLog2e);
+        s_edge *= scale;
 #pragma unroll
-      for (int i = 0; i < H; ++i) { s2[i] = make_float2(0.f, 0.f); zs2[i] = make_float2(0.f, 0.f); }
-      float acc[2] = {0.f, 0.f};
-      for (int k = 0; k < n_pieces; ++k) {
+        for (int i = 0; i < H; ++i) s2[i] = __fmul2_rn(s2[i], scale2);
 #pragma unroll
         for (int u = 0; u < kSegPerThread; ++u) {
           const int s = k * kSegPerChunk + u * kConsumers + tid;
-          if (s >= g.seg_lo && s < g.seg_hi) {
+          if (inner[u]) {
             float2 z2[H];
-            SegOps<T>::unpack2(*reinterpret_cast<const uint4*>(img + (size_t)s * 16), z2);
+            SegOps<T>::unpack2(raw[u], z2);
 #pragma unroll
             for (int i = 0; i < H; ++i) {
-              s2[i] = __fadd2_rn(s2[i], exp_shift2<T>(z2[i], m, l2e2, nml2));
+              s2[i] = __fadd2_rn(s2[i], exp_shift2<T>(z2[i], best, l2e2, nml2k));
               zs2[i] = __fadd2_rn(zs2[i], z2[i]);
             }
-          } else if (s < g.n_seg) {
+          } else if (ragged[u]) {
             float z[V];
-            SegOps<T>::unpack(*reinterpret_cast<const uint4*>(img + (size_t)s * 16), z);
+            SegOps<T>::unpack(raw[u], z);
 #pragma unroll
             for (int i = 0; i < V; ++i) {
               const int64_t c = (int64_t)s * V - g.head + i;
               if (c >= 0 && c < C) {
-                acc[0] += exp_shift2<T>(make_float2(z[i], z[i]), m, l2e2, nml2).x;
-                acc[1] += z[i];
+                s_edge += exp_shift2<T>(make_float2(z[i], z[i]), best, l2e2, nml2k).x;
+                z_edge += z[i];
               }
             }
           }
         }
       }
+      float s_t = s_edge, z_t = z_edge;
 #pragma unroll
-      for (int i = 0; i < H; ++i) { acc[0] += s2[i].x + s2[i].y; acc[1] += zs2[i].x + zs2[i].y; }
-      red.sum(acc);
-      const float S = acc[0], sum_z = acc[1];
+      for (int i = 0; i < H; ++i) { s_t += s2[i].x + s2[i].y; z_t += zs2[i].x + zs2[i].y; }
+      // block reduction in one round: maximum with its first segment, then the sums rescaled to it
+      float m = best;
+      int m_seg = best_seg;
+      float S, sum_z;
+      {
+        warp_argmax(m, m_seg);
+        float sw = warp_sum(s_t * rescale_exp2<T>((best - m) * kLog2e));
+        float zw = warp_sum(z_t);
+        float* sc = ctrl->red[red.toggle];
+        if (lane == 0) {
+          sc[red.warp] = m;
+          reinterpret_cast<int*>(sc)[NCW + red.warp] = m_seg;
+          sc[2 * NCW + red.warp] = sw;
+          sc[3 * NCW + red.warp] = zw;
+        }
+        ConsumerReduce<NCW>::bar();
+        const float mw = lane < NCW ? sc[lane] : -3.0e38f;
+        int segw = lane < NCW ? reinterpret_cast<int*>(sc)[NCW + lane] : 0x7fffffff;
+        const float sws = lane < NCW ? sc[2 * NCW + lane] : 0.f;
+        const float zws = lane < NCW ? sc[3 * NCW + lane] : 0.f;
+        m = mw;
+        m_seg = segw;
+        warp_argmax(m, m_seg);
+        S = warp_sum(sws * rescale_exp2<T>((mw - m) * kLog2e));
+        sum_z = warp_sum(zws);
+        red.toggle ^= 1;
+      }
+      if (m_seg >= g.n_seg) m_seg = 0;  // NaN rows: keep the read below inside the row image
+      const float2 nml2 = make_float2(-m * kLog2e, -m * kLog2e);
+      // every thread reads the winning segment: first column that attains the maximum
+      const int a_own = first_equal<T>(img, m_seg, g.head, C, m);
+      const int seg_a = a.want_flags ? m_seg : -1;
       const float zy = Elem<T>::to_f32(reinterpret_cast<const T*>(img)[g.head + y]);
       const float ce = (m + logf(S)) - (1.f - a.eps) * zy - (a.eps / (float)C) * sum_z;
 
@@ -749,8 +839,10 @@ rows_tma_kernel(const __grid_constant__ KArgs a, const TmaCfg cfg) {
       }
       ++v;
 
-      // ---------------- row results: one merged reduction that only consumer warp 0 waits for
+      // ---------------- row results: per-warp partials go to the service warp, nobody waits here
       {
+        const int par = (v - 1) & 1;  // v was advanced above
+        const int done = v - 1;       // index of this valid row
         float part[1 + 3 * PD];
         part[0] = warp_sum(dist2.x + dist2.y);
 #pragma unroll
@@ -759,34 +851,13 @@ rows_tma_kernel(const __grid_constant__ KArgs a, const TmaCfg cfg) {
           part[2 + 3 * j] = warp_max(SegOps<T>::to_float(ge[j]));
           part[3 + 3 * j] = warp_max(za[j]);
         }
-        const int cw = warp - 2;
+        if (done >= 2) wait_bounded(&ctrl->end_empty[par], (uint32_t)((done >> 1) - 1) & 1u, ctrl, a.hdr);
         if (lane == 0) {
+          const int cw = red.warp;
 #pragma unroll
-          for (int i = 0; i < 1 + 3 * PD; ++i) ctrl->endred[i * NCW + cw] = part[i];
-        }
-        __threadfence_block();
-        if (cw != 0) {
-          asm volatile("bar.arrive 2, %0;" ::"n"(NCW * 32) : "memory");
-        } else {
-          asm volatile("bar.sync 2, %0;" ::"n"(NCW * 32) : "memory");
-          float dsum = warp_sum(lane < NCW ? ctrl->endred[lane] : 0.f);
-          uint32_t flags = 0u;
-          if (a.want_flags) {
-            flags = (a_own == y) ? 1u : 0u;
-#pragma unroll
-            for (int j = 0; j < P; ++j) {
-              const float ltv = warp_max(lane < NCW ? ctrl->endred[(1 + 3 * j) * NCW + lane] : -INFINITY);
-              const float gev = warp_max(lane < NCW ? ctrl->endred[(2 + 3 * j) * NCW + lane] : -INFINITY);
-              const float zav = warp_max(lane < NCW ? ctrl->endred[(3 + 3 * j) * NCW + lane] : -INFINITY);
-              if (zav >= gev && ltv < zav) flags |= (2u << j);
-            }
-          }
-          if (lane == 0) {
-            float D = 0.f;
-            if (with_term) D = PW ? dsum * inv_P / (float)C : dsum * inv_P * inv_P / (float)C;
-            a.row_loss[r] = with_term ? fmaf(a.alpha, D, ce) : ce;
-            a.row_flags[r] = flags;
-          }
+          for (int i = 0; i < 1 + 3 * PD; ++i) ctrl->endred[par][i * NCW + cw] = part[i];
+          if (cw == 0) { ctrl->end_ce[par] = ce; ctrl->end_correct[par] = (a_own == y); }
+          mbar_arrive(&ctrl->end_full[par]);
         }
       }
     }
