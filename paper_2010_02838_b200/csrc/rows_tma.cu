@@ -598,6 +598,19 @@ rows_tma_kernel(const __grid_constant__ KArgs a, const TmaCfg cfg) {
       char* g_img = a.grad ? reinterpret_cast<char*>(a.grad) + lr * a.row_stride * ES - (int64_t)g.head * ES : nullptr;
 
       if (!valid) continue;  // masked rows are written by the service warp
+      // Bit k set: in piece k this thread has a segment that needs care (ragged edge of the row, or
+      // past its end); all other pieces take straight-line code.
+      uint32_t odd_sweep = 0u;
+      {
+        auto mark = [&](int s) {
+          if (((s % kSegPerChunk) % kConsumers) == tid) odd_sweep |= 1u << (s / kSegPerChunk);
+        };
+        if (g.seg_lo > 0) mark(0);
+        if (g.seg_hi < g.n_seg) mark(g.n_seg - 1);
+        const int room = g.n_seg - (kSegPerThread - 1) * kConsumers - tid;  // segments before this thread's last lane runs out
+        const int k_bad = room > 0 ? (room + kSegPerChunk - 1) / kSegPerChunk : 0;
+        if (k_bad < 32) odd_sweep |= ~0u << k_bad;
+      }
       const uint32_t own_parity = (uint32_t)v & 1u;
 
       // ---------------- one sweep over the own row, piece by piece as it lands (online softmax):
@@ -612,6 +625,35 @@ rows_tma_kernel(const __grid_constant__ KArgs a, const TmaCfg cfg) {
       float s_edge = 0.f, z_edge = 0.f;  // contributions of ragged edge segments (relative to `best`)
       for (int k = 0; k < n_pieces; ++k) {
         wait_bounded(&ctrl->own_full[k], own_parity, ctrl, a.hdr);
+        if (!((odd_sweep >> k) & 1u)) {
+          // ---- straight-line path: all of this thread's segments of the piece lie inside the row
+          const uint32_t off = (uint32_t)k * kChunkBytes + (uint32_t)tid * 16u;
+          uint4 rw[kSegPerThread];
+          const float old_best = best;
+#pragma unroll
+          for (int u = 0; u < kSegPerThread; ++u) {
+            rw[u] = *reinterpret_cast<const uint4*>(img + off + u * (kConsumers * 16));
+            const float fm = SegOps<T>::to_float(SegOps<T>::fold(rw[u]));
+            if (fm > best) { best = fm; best_seg = k * kSegPerChunk + u * kConsumers + tid; }
+          }
+          const float sc = rescale_exp2<T>((old_best - best) * kLog2e);
+          const float2 sc2 = make_float2(sc, sc);
+          const float2 nmk = make_float2(-best * kLog2e, -best * kLog2e);
+          s_edge *= sc;
+#pragma unroll
+          for (int i = 0; i < H; ++i) s2[i] = __fmul2_rn(s2[i], sc2);
+#pragma unroll
+          for (int u = 0; u < kSegPerThread; ++u) {
+            float2 z2[H];
+            SegOps<T>::unpack2(rw[u], z2);
+#pragma unroll
+            for (int i = 0; i < H; ++i) {
+              s2[i] = __fadd2_rn(s2[i], exp_shift2<T>(z2[i], best, l2e2, nmk));
+              zs2[i] = __fadd2_rn(zs2[i], z2[i]);
+            }
+          }
+          continue;
+        }
         uint4 raw[kSegPerThread];
         bool inner[kSegPerThread], ragged[kSegPerThread];
         const float old = best;
@@ -719,7 +761,66 @@ rows_tma_kernel(const __grid_constant__ KArgs a, const TmaCfg cfg) {
 #pragma unroll
       for (int j = 0; j < PD; ++j) { lt[j] = SegOps<T>::neg_inf(); ge[j] = SegOps<T>::neg_inf(); za[j] = -INFINITY; }
 
+      // pieces that also hold the arg-max column or the label column are handled by the general code
+      uint32_t odd = odd_sweep;
+      if (((seg_y % kSegPerChunk) % kConsumers) == tid) odd |= 1u << (seg_y / kSegPerChunk);
+      if (seg_a >= 0 && ((seg_a % kSegPerChunk) % kConsumers) == tid) odd |= 1u << (seg_a / kSegPerChunk);
+      const bool lean_ok = with_term && a.want_flags && g_img != nullptr;
+      float2 dist2b = make_float2(0.f, 0.f);
+      const uint32_t tid16 = (uint32_t)tid * 16u;
+
       for (int k = 0; k < n_pieces; ++k) {
+        if (lean_ok && !((odd >> k) & 1u)) {
+          // ---- straight-line path: every segment of this thread lies inside the row, away from the
+          // arg-max and label columns
+          const uint32_t off = (uint32_t)k * kChunkBytes + tid16;
+          float2 z2[kSegPerThread][H], sd2[kSegPerThread][H];
+          bool before[kSegPerThread];
+#pragma unroll
+          for (int u = 0; u < kSegPerThread; ++u) {
+            SegOps<T>::unpack2(*reinterpret_cast<const uint4*>(img + off + u * (kConsumers * 16)), z2[u]);
+            before[u] = (k * kSegPerChunk + u * kConsumers + tid) < seg_a;
+          }
+#pragma unroll
+          for (int j = 0; j < P; ++j) {
+            wait_bounded(&ctrl->ring_full[st], st_phase, ctrl, a.hdr);
+            const char* chunk = ring_base + (uint32_t)st * kChunkBytes + tid16;
+            uint4 raw[kSegPerThread];
+#pragma unroll
+            for (int u = 0; u < kSegPerThread; ++u) raw[u] = *reinterpret_cast<const uint4*>(chunk + u * (kConsumers * 16));
+#pragma unroll
+            for (int u = 0; u < kSegPerThread; ++u) {
+              float2 v2[H];
+              SegOps<T>::unpack2(raw[u], v2);
+#pragma unroll
+              for (int i = 0; i < H; ++i) {
+                const float2 d = __ffma2_rn(v2[i], neg1, z2[u][i]);
+                if (P == 1 || j == 0) sd2[u][i] = d; else sd2[u][i] = __fadd2_rn(sd2[u][i], d);
+                if constexpr (PW) { if (i & 1) dist2b = __ffma2_rn(d, d, dist2b); else dist2 = __ffma2_rn(d, d, dist2); }
+              }
+              const typename SegOps<T>::macc f = SegOps<T>::fold(raw[u]);
+              lt[j] = before[u] ? SegOps<T>::mmax(lt[j], f) : lt[j];
+              ge[j] = before[u] ? ge[j] : SegOps<T>::mmax(ge[j], f);
+            }
+            __syncwarp();
+            if (lane == 0) mbar_arrive(&ctrl->ring_empty[st]);
+            if (++st == n_stage) { st = 0; st_phase ^= 1u; }
+          }
+#pragma unroll
+          for (int u = 0; u < kSegPerThread; ++u) {
+            float2 g2[H];
+#pragma unroll
+            for (int i = 0; i < H; ++i) {
+              const float2 e = exp_shift2<T>(z2[u][i], m, l2e2, nml2);
+              g2[i] = __ffma2_rn(e, cp2, __ffma2_rn(sd2[u][i], cd2, ncq2));
+              if constexpr (!PW) dist2 = __ffma2_rn(sd2[u][i], sd2[u][i], dist2);
+            }
+            *reinterpret_cast<uint4*>(g_img + off + u * (kConsumers * 16)) = SegOps<T>::pack2(g2);
+          }
+          __syncwarp();
+          if (lane == 0) mbar_arrive(&ctrl->own_empty[k]);
+          continue;
+        }
         float2 z2[kSegPerThread][H], sd2[kSegPerThread][H];
         bool active[kSegPerThread], special[kSegPerThread], edge[kSegPerThread];
         int seg[kSegPerThread];
@@ -844,7 +945,7 @@ rows_tma_kernel(const __grid_constant__ KArgs a, const TmaCfg cfg) {
         const int par = (v - 1) & 1;  // v was advanced above
         const int done = v - 1;       // index of this valid row
         float part[1 + 3 * PD];
-        part[0] = warp_sum(dist2.x + dist2.y);
+        part[0] = warp_sum((dist2.x + dist2.y) + (dist2b.x + dist2b.y));
 #pragma unroll
         for (int j = 0; j < PD; ++j) {
           part[1 + 3 * j] = warp_max(SegOps<T>::to_float(lt[j]));
