@@ -65,7 +65,7 @@ struct Ctrl {  // lives at the start of dynamic shared memory
   int last_flag;
   uint64_t end_full[2];    // consumers -> service warp: partial results of a row are in endred[par]
   uint64_t end_empty[2];   // service warp -> consumers: endred[par] may be overwritten
-  float red[2][kMaxConsumerWarps * 4];      // reduction scratch of the consumers, two alternating halves
+  alignas(16) float red[2][kMaxConsumerWarps * 4];  // reduction scratch of the consumers, two alternating halves
   float endred[2][kMaxConsumerWarps * 24];  // per-warp partials of the end-of-row reduction
   float end_ce[2];                          // task loss of the row
   int end_correct[2];                       // arg-max == label
@@ -213,6 +213,15 @@ __device__ __forceinline__ float2 exp_shift2(float2 z, float m, float2 l2e, floa
 template <typename T>
 __device__ __forceinline__ float rescale_exp2(float x) {
   if constexpr (sizeof(T) == 4) return exp2f(x); else return ex2_approx(x);
+}
+
+// Order-preserving map between floats and unsigned integers (for integer warp reductions).
+__device__ __forceinline__ unsigned float_order_key(float f) {
+  const unsigned u = __float_as_uint(f);
+  return (u & 0x80000000u) ? ~u : (u | 0x80000000u);
+}
+__device__ __forceinline__ float float_from_order_key(unsigned k) {
+  return __uint_as_float((k & 0x80000000u) ? (k & 0x7fffffffu) : ~k);
 }
 
 // Geometry of one row image.
@@ -717,26 +726,33 @@ rows_tma_kernel(const __grid_constant__ KArgs a, const TmaCfg cfg) {
       int m_seg = best_seg;
       float S, sum_z;
       {
-        warp_argmax(m, m_seg);
-        float sw = warp_sum(s_t * rescale_exp2<T>((best - m) * kLog2e));
-        float zw = warp_sum(z_t);
-        float* sc = ctrl->red[red.toggle];
-        if (lane == 0) {
-          sc[red.warp] = m;
-          reinterpret_cast<int*>(sc)[NCW + red.warp] = m_seg;
-          sc[2 * NCW + red.warp] = sw;
-          sc[3 * NCW + red.warp] = zw;
-        }
+        // within the warp: the maximum by an integer reduction on an order-preserving image of the
+        // float (-0 is folded onto +0 first: they tie), its first segment by a second one; the sums
+        // by shuffles
+        const unsigned key = float_order_key(best + 0.f);
+        const unsigned key_w = __reduce_max_sync(0xffffffffu, key);
+        const int seg_w = (int)__reduce_min_sync(0xffffffffu, key == key_w ? (unsigned)best_seg : 0x7fffffffu);
+        const float m_w = float_from_order_key(key_w);
+        const float sw = warp_sum(s_t * rescale_exp2<T>((best - m_w) * kLog2e));
+        const float zw = warp_sum(z_t);
+        float4* sc = reinterpret_cast<float4*>(ctrl->red[red.toggle]);
+        if (lane == 0) sc[red.warp] = make_float4(m_w, __int_as_float(seg_w), sw, zw);
         ConsumerReduce<NCW>::bar();
-        const float mw = lane < NCW ? sc[lane] : -3.0e38f;
-        int segw = lane < NCW ? reinterpret_cast<int*>(sc)[NCW + lane] : 0x7fffffff;
-        const float sws = lane < NCW ? sc[2 * NCW + lane] : 0.f;
-        const float zws = lane < NCW ? sc[3 * NCW + lane] : 0.f;
-        m = mw;
-        m_seg = segw;
-        warp_argmax(m, m_seg);
-        S = warp_sum(sws * rescale_exp2<T>((mw - m) * kLog2e));
-        sum_z = warp_sum(zws);
+        // across warps: every thread combines the NCW partials itself (broadcast reads, fixed order)
+        float4 part[NCW];
+#pragma unroll
+        for (int wv = 0; wv < NCW; ++wv) part[wv] = sc[wv];
+        m = part[0].x;
+        m_seg = __float_as_int(part[0].y);
+#pragma unroll
+        for (int wv = 1; wv < NCW; ++wv) argmax_combine(m, m_seg, part[wv].x, __float_as_int(part[wv].y));
+        S = 0.f;
+        sum_z = 0.f;
+#pragma unroll
+        for (int wv = 0; wv < NCW; ++wv) {
+          S += part[wv].z * rescale_exp2<T>((part[wv].x - m) * kLog2e);
+          sum_z += part[wv].w;
+        }
         red.toggle ^= 1;
       }
       if (m_seg >= g.n_seg) m_seg = 0;  // NaN rows: keep the read below inside the row image
