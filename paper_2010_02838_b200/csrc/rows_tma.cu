@@ -2,17 +2,17 @@
 //
 // Each CTA owns one resident row buffer and a ring of stages; as many CTAs as fit run per SM (two
 // for 64 KiB rows), so that one CTA's statistics pass overlaps the other's streaming pass.
-//   warp 0  scheduler + own-row producer: draws row ids from a global counter (mask byte and label
-//           are fetched one row ahead), publishes them in a small ring of row-info slots, and moves
-//           the own row image into the row buffer piece by piece with 1-D bulk asynchronous copies
-//           (cp.async.bulk, no multicast) that complete on one mbarrier per piece.  A piece is
-//           refilled for the next row as soon as the consumers are done with it, so the next own
-//           row streams in behind the current row's second pass.
+//   warp 0  scheduler + own-row producer + service: draws row ids from a global counter (mask byte
+//           and label are fetched one row ahead), publishes them in a small ring of row-info slots,
+//           and moves the own row image into the row buffer piece by piece with 1-D bulk
+//           asynchronous copies (cp.async.bulk, no multicast) that complete on one mbarrier per
+//           piece.  A piece is refilled for the next row as soon as the consumers are done with it,
+//           so the next own row streams in behind the current row's second pass.  The same warp
+//           writes the all-zero gradient rows of masked rows and turns the consumers' per-warp
+//           partial results of a finished row into the per-row loss and flag word, off the
+//           consumers' critical path.
 //   warp 1  peer producer: streams the n-1 peer rows chunk by chunk (chunk-major: chunk k of peer
 //           0, 1, ..., then chunk k+1) through the ring of stages.
-//   warp 2  service warp: writes the all-zero gradient rows of masked rows and turns the consumers'
-//           per-warp partial results of a finished row into the per-row loss and flag word, off
-//           the consumers' critical path.
 //   others  consumers: one sweep over the resident own row as its pieces land (online softmax:
 //           running max, sum exp, sum z, first arg-max), one block reduction, then per chunk:
 //           consume the peers from the ring (sum_j (z - z_j), sum_j (z - z_j)^2, what the arg-max
@@ -451,46 +451,6 @@ rows_tma_kernel(const __grid_constant__ KArgs a, const TmaCfg cfg) {
       t_next2 = a.row_begin + (long long)atomicAdd(&a.hdr->next_row, 1u);
       if (t_next < a.row_end) { mask_next = a.mask ? a.mask[t_next] : 1; label_next = a.labels[t_next]; }
     }
-    int v = 0;  // valid rows copied so far
-    for (int it = 0;; ++it) {
-      long long r = t_next;
-      int mask_v = mask_next, label_v = label_next;
-      if (lane == 0) {
-        t_next = t_next2;
-        t_next2 = a.row_begin + (long long)atomicAdd(&a.hdr->next_row, 1u);
-        if (t_next < a.row_end) { mask_next = a.mask ? a.mask[t_next] : 1; label_next = a.labels[t_next]; }
-      }
-      r = __shfl_sync(0xffffffffu, r, 0);
-      mask_v = __shfl_sync(0xffffffffu, mask_v, 0);
-      label_v = __shfl_sync(0xffffffffu, label_v, 0);
-      const bool more = r < a.row_end;
-      const bool valid = more && mask_v != 0 && label_v >= 0 && (int64_t)label_v < C;
-      const int slot = it % kInfoSlots;
-      if (it >= kInfoSlots) wait_bounded(&ctrl->info_empty[slot], ((it / kInfoSlots) - 1) & 1, ctrl, a.hdr);
-      if (lane == 0) {
-        ctrl->info[slot].row = more ? r : -1;
-        ctrl->info[slot].valid = valid;
-        ctrl->info[slot].label = label_v;
-        mbar_arrive(&ctrl->info_full[slot]);
-      }
-      if (!more) break;
-      if (!valid) continue;
-      const RowCopy rc = row_copy<T>(a, r);
-      const char* src = reinterpret_cast<const char*>(a.own) + rc.row_off;
-      for (int k = 0; k < n_pieces; ++k) {
-        if (v >= 1) wait_bounded(&ctrl->own_empty[k], (v - 1) & 1, ctrl, a.hdr);
-        const uint32_t begin = (uint32_t)k * kChunkBytes;
-        uint32_t end = begin + kChunkBytes < rc.img_bytes ? begin + kChunkBytes : rc.img_bytes;
-        if (end < begin) end = begin;  // empty piece of a shorter row image
-        produce_copy<T>(own_buf + begin, src, begin, end, rc.tma_limit, rc.valid_end, &ctrl->own_full[k], lane);
-      }
-      ++v;
-    }
-    // Before leaving, make sure no copy armed by this warp is still in flight (bounded).
-    if (v >= 1)
-      for (int k = 0; k < n_pieces; ++k) wait_bounded(&ctrl->own_full[k], (v - 1) & 1, ctrl, a.hdr);
-  } else if (warp == 1) {
-    // ============================== peer producer + service ==============================
     const float inv_P = P >= 1 ? 1.f / (float)P : 0.f;
     // Turns the consumers' per-warp partials of valid row number `vv` into its loss and flag word.
     auto finish_row = [&](int vv, long long row) {
@@ -519,19 +479,30 @@ rows_tma_kernel(const __grid_constant__ KArgs a, const TmaCfg cfg) {
         a.row_flags[row] = flags;
       }
     };
-    uint32_t q = 0;          // ring items issued so far
-    int st = 0;              // stage of the next item
-    uint32_t st_phase = 0;   // phase bit of that stage's next use
-    int v = 0;               // valid rows seen so far
+    int v = 0;  // valid rows copied so far
     long long prev_row[2] = {-1, -1};  // rows whose results are still to be finished (valid rows v-2, v-1)
     for (int it = 0;; ++it) {
+      long long r = t_next;
+      int mask_v = mask_next, label_v = label_next;
+      if (lane == 0) {
+        t_next = t_next2;
+        t_next2 = a.row_begin + (long long)atomicAdd(&a.hdr->next_row, 1u);
+        if (t_next < a.row_end) { mask_next = a.mask ? a.mask[t_next] : 1; label_next = a.labels[t_next]; }
+      }
+      r = __shfl_sync(0xffffffffu, r, 0);
+      mask_v = __shfl_sync(0xffffffffu, mask_v, 0);
+      label_v = __shfl_sync(0xffffffffu, label_v, 0);
+      const bool more = r < a.row_end;
+      const bool valid = more && mask_v != 0 && label_v >= 0 && (int64_t)label_v < C;
       const int slot = it % kInfoSlots;
-      wait_bounded(&ctrl->info_full[slot], (it / kInfoSlots) & 1, ctrl, a.hdr);
-      const long long r = ctrl->info[slot].row;
-      const bool valid = ctrl->info[slot].valid != 0;
-      __syncwarp();
-      if (lane == 0) mbar_arrive(&ctrl->info_empty[slot]);
-      if (r < 0) break;
+      if (it >= kInfoSlots) wait_bounded(&ctrl->info_empty[slot], ((it / kInfoSlots) - 1) & 1, ctrl, a.hdr);
+      if (lane == 0) {
+        ctrl->info[slot].row = more ? r : -1;
+        ctrl->info[slot].valid = valid;
+        ctrl->info[slot].label = label_v;
+        mbar_arrive(&ctrl->info_full[slot]);
+      }
+      if (!more) break;
       if (!valid) {  // masked row: zero gradient, no loss, no counts; nothing is copied for it
         if (a.grad) {
           const int64_t lr = r - a.row_begin;
@@ -556,8 +527,37 @@ rows_tma_kernel(const __grid_constant__ KArgs a, const TmaCfg cfg) {
       // before feeding row v (the consumers reuse its partial-result slot at the end of row v).
       if (v >= 2) finish_row(v - 2, prev_row[v & 1]);
       prev_row[v & 1] = r;
+      const RowCopy rc = row_copy<T>(a, r);
+      const char* src = reinterpret_cast<const char*>(a.own) + rc.row_off;
+      for (int k = 0; k < n_pieces; ++k) {
+        if (v >= 1) wait_bounded(&ctrl->own_empty[k], (v - 1) & 1, ctrl, a.hdr);
+        const uint32_t begin = (uint32_t)k * kChunkBytes;
+        uint32_t end = begin + kChunkBytes < rc.img_bytes ? begin + kChunkBytes : rc.img_bytes;
+        if (end < begin) end = begin;  // empty piece of a shorter row image
+        produce_copy<T>(own_buf + begin, src, begin, end, rc.tma_limit, rc.valid_end, &ctrl->own_full[k], lane);
+      }
       ++v;
-      if (!stream_peers) continue;
+    }
+    // results of the last two valid rows
+    if (v >= 2) finish_row(v - 2, prev_row[v & 1]);
+    if (v >= 1) finish_row(v - 1, prev_row[(v - 1) & 1]);
+    // Before leaving, make sure no copy armed by this warp is still in flight (bounded).
+    if (v >= 1)
+      for (int k = 0; k < n_pieces; ++k) wait_bounded(&ctrl->own_full[k], (v - 1) & 1, ctrl, a.hdr);
+  } else if (warp == 1) {
+    // ============================== peer producer ==============================
+    uint32_t q = 0;          // ring items issued so far
+    int st = 0;              // stage of the next item
+    uint32_t st_phase = 0;   // phase bit of that stage's next use
+    for (int it = 0;; ++it) {
+      const int slot = it % kInfoSlots;
+      wait_bounded(&ctrl->info_full[slot], (it / kInfoSlots) & 1, ctrl, a.hdr);
+      const long long r = ctrl->info[slot].row;
+      const bool valid = ctrl->info[slot].valid != 0;
+      __syncwarp();
+      if (lane == 0) mbar_arrive(&ctrl->info_empty[slot]);
+      if (r < 0) break;
+      if (!valid || !stream_peers) continue;
       const RowCopy rc = row_copy<T>(a, r);
       for (int k = 0; k < n_pieces; ++k) {
         const uint32_t begin = (uint32_t)k * kChunkBytes;
@@ -572,9 +572,6 @@ rows_tma_kernel(const __grid_constant__ KArgs a, const TmaCfg cfg) {
         }
       }
     }
-    // results of the last two valid rows
-    if (v >= 2) finish_row(v - 2, prev_row[v & 1]);
-    if (v >= 1) finish_row(v - 1, prev_row[(v - 1) & 1]);
     for (uint32_t i = 0; i < (uint32_t)n_stage && i < q; ++i) {
       const uint32_t qi = q - 1 - i;
       wait_bounded(&ctrl->ring_full[qi % n_stage], (qi / n_stage) & 1, ctrl, a.hdr);
