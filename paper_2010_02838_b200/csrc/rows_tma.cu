@@ -110,8 +110,8 @@ __device__ __forceinline__ unsigned long long global_timer_ns() {
 
 // Wait for a phase of an mbarrier, but never for ever: after kWaitLimitNs the CTA-wide abort flag
 // and the device status are set and every later wait returns at once (results are then invalid).
-__device__ __forceinline__ void wait_bounded(uint64_t* bar, uint32_t parity, Ctrl* ctrl, WsHeader* hdr) {
-  if (mbar_try_wait(bar, parity)) return;
+// The polling loop is kept out of line so that the callers' code stays compact.
+__device__ __noinline__ void wait_slow(uint64_t* bar, uint32_t parity, Ctrl* ctrl, WsHeader* hdr) {
   volatile int* abort_flag = &ctrl->abort_flag;
   uint32_t polls = 0;
   unsigned long long t0 = 0;
@@ -128,6 +128,10 @@ __device__ __forceinline__ void wait_bounded(uint64_t* bar, uint32_t parity, Ctr
       }
     }
   }
+}
+__device__ __forceinline__ void wait_bounded(uint64_t* bar, uint32_t parity, Ctrl* ctrl, WsHeader* hdr) {
+  if (mbar_try_wait(bar, parity)) return;
+  wait_slow(bar, parity, ctrl, hdr);
 }
 
 // ------------------------------------------------------------------ 16-byte segments
