@@ -361,7 +361,7 @@ __device__ __forceinline__ RowCopy row_copy(const KArgs& a, long long r) {
 
 // First column of segment `s` whose value equals m, or INT_MAX.
 template <typename T>
-__device__ __forceinline__ int first_equal(const char* img, int s, int head, int64_t C, float m) {
+__device__ __noinline__ int first_equal(const char* img, int s, int head, int64_t C, float m) {
   constexpr int V = SegOps<T>::V;
   float z[V];
   SegOps<T>::unpack(*reinterpret_cast<const uint4*>(img + (size_t)s * 16), z);
