@@ -30,7 +30,8 @@ namespace codistill {
 constexpr int kMaxStages = 12;
 constexpr int kMaxPieces = 32;
 constexpr int kInfoSlots = 4;
-constexpr int kCtrlBytes = 6144;
+constexpr int kCtrlBytes = 8192;        // control block, then kZeroBytes of zeros
+constexpr int kZeroBytes = 2048;        // source of the bulk stores that write all-zero gradient rows
 constexpr int kProducerThreads = 64;   // warp 0: scheduler + own row, warp 1: peers + service
 constexpr int kSegPerThread = 2;       // 16-byte segments per consumer thread per chunk
 constexpr int kMaxConsumerWarps = 16;
@@ -71,7 +72,7 @@ struct Ctrl {  // lives at the start of dynamic shared memory
   int end_correct[2];                       // arg-max == label
   double fin[32];
 };
-static_assert(sizeof(Ctrl) <= kCtrlBytes, "control block fits its slot");
+static_assert(sizeof(Ctrl) <= kCtrlBytes - kZeroBytes, "control block fits its slot");
 
 // ------------------------------------------------------------------ PTX wrappers
 __device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
@@ -101,6 +102,11 @@ __device__ __forceinline__ void bulk_g2s(void* dst, const void* src, uint32_t by
                    smem_u32(dst)),
                "l"(src), "r"(bytes), "r"(smem_u32(bar))
                : "memory");
+}
+// shared -> global bulk copy; dst, src and bytes are multiples of 16.  Completion is tracked by the
+// issuing thread's bulk async-group.
+__device__ __forceinline__ void bulk_s2g(void* dst, const void* src, uint32_t bytes) {
+  asm volatile("cp.async.bulk.global.shared::cta.bulk_group [%0], [%1], %2;" ::"l"(dst), "r"(smem_u32(src)), "r"(bytes) : "memory");
 }
 __device__ __forceinline__ unsigned long long global_timer_ns() {
   unsigned long long t;
@@ -442,6 +448,9 @@ rows_tma_kernel(const __grid_constant__ KArgs a, const TmaCfg cfg) {
     ctrl->last_flag = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
+  char* zero_region = reinterpret_cast<char*>(smem_raw) + (kCtrlBytes - kZeroBytes);
+  for (int i = threadIdx.x * 16; i < kZeroBytes; i += blockDim.x * 16) *reinterpret_cast<uint4*>(zero_region + i) = make_uint4(0u, 0u, 0u, 0u);
+  asm volatile("fence.proxy.async.shared::cta;" ::: "memory");  // the zeros are read by bulk copies later
   __syncthreads();
 
   if (warp == 0) {
@@ -509,13 +518,18 @@ rows_tma_kernel(const __grid_constant__ KArgs a, const TmaCfg cfg) {
       if (!more) break;
       if (!valid) {  // masked row: zero gradient, no loss, no counts; nothing is copied for it
         if (a.grad) {
+          // whole segments inside the row: bulk copies of zeros; the ragged first / last segments: element stores
           const int64_t lr = r - a.row_begin;
           const RowGeom g = row_geom<T>(lr, a.row_stride, C);
           char* g_img = reinterpret_cast<char*>(a.grad) + lr * a.row_stride * ES - (int64_t)g.head * ES;
-          for (int s = lane; s < g.n_seg; s += 32) {
-            if (s >= g.seg_lo && s < g.seg_hi) {
-              *reinterpret_cast<uint4*>(g_img + (size_t)s * 16) = make_uint4(0u, 0u, 0u, 0u);
-            } else {
+          if (lane == 0) {
+            const uint32_t lo = (uint32_t)g.seg_lo * 16u, hi = (uint32_t)g.seg_hi * 16u;
+            for (uint32_t o = lo; o < hi; o += kZeroBytes) bulk_s2g(g_img + o, zero_region, hi - o < (uint32_t)kZeroBytes ? hi - o : (uint32_t)kZeroBytes);
+            asm volatile("cp.async.bulk.commit_group;" ::: "memory");
+          }
+          if (lane < 2) {
+            const int s = lane == 0 ? 0 : g.n_seg - 1;
+            if ((lane == 0 && g.seg_lo > 0) || (lane == 1 && g.seg_hi < g.n_seg && (g.n_seg > 1 || g.seg_lo == 0))) {
 #pragma unroll
               for (int i = 0; i < V; ++i) {
                 const int64_t c = (int64_t)s * V - g.head + i;
@@ -545,6 +559,7 @@ rows_tma_kernel(const __grid_constant__ KArgs a, const TmaCfg cfg) {
     // results of the last two valid rows
     if (v >= 2) finish_row(v - 2, prev_row[v & 1]);
     if (v >= 1) finish_row(v - 1, prev_row[(v - 1) & 1]);
+    if (lane == 0) asm volatile("cp.async.bulk.wait_group 0;" ::: "memory");  // zero rows are written
     // Before leaving, make sure no copy armed by this warp is still in flight (bounded).
     if (v >= 1)
       for (int k = 0; k < n_pieces; ++k) wait_bounded(&ctrl->own_full[k], (v - 1) & 1, ctrl, a.hdr);
@@ -778,10 +793,13 @@ rows_tma_kernel(const __grid_constant__ KArgs a, const TmaCfg cfg) {
 #pragma unroll
       for (int j = 0; j < PD; ++j) { lt[j] = SegOps<T>::neg_inf(); ge[j] = SegOps<T>::neg_inf(); za[j] = -INFINITY; }
 
-      // pieces that also hold the arg-max column or the label column are handled by the general code
-      uint32_t odd = odd_sweep;
-      if (((seg_y % kSegPerChunk) % kConsumers) == tid) odd |= 1u << (seg_y / kSegPerChunk);
-      if (seg_a >= 0 && ((seg_a % kSegPerChunk) % kConsumers) == tid) odd |= 1u << (seg_a / kSegPerChunk);
+      // The thread that holds the label column or the own arg-max column patches its straight-line
+      // code for that one segment (bit k of spec_y / spec_a: it is in piece k); only ragged pieces
+      // take the general code.
+      const uint32_t odd = odd_sweep;
+      const uint32_t spec_y = (((seg_y % kSegPerChunk) % kConsumers) == tid) ? 1u << (seg_y / kSegPerChunk) : 0u;
+      const uint32_t spec_a = (seg_a >= 0 && ((seg_a % kSegPerChunk) % kConsumers) == tid) ? 1u << (seg_a / kSegPerChunk) : 0u;
+      const int u_y = (seg_y % kSegPerChunk) / kConsumers, u_a = seg_a >= 0 ? (seg_a % kSegPerChunk) / kConsumers : 0;
       const bool lean_ok = with_term && a.want_flags && g_img != nullptr;
       float2 dist2b = make_float2(0.f, 0.f);
       const uint32_t tid16 = (uint32_t)tid * 16u;
@@ -819,6 +837,21 @@ rows_tma_kernel(const __grid_constant__ KArgs a, const TmaCfg cfg) {
               lt[j] = before[u] ? SegOps<T>::mmax(lt[j], f) : lt[j];
               ge[j] = before[u] ? ge[j] : SegOps<T>::mmax(ge[j], f);
             }
+            if ((spec_a >> k) & 1u) {
+              // The segment of the own arg-max column a went to ge[] as a whole.  The peer's value at a and
+              // the largest value before a inside the segment settle the rest: with them in za[] and lt[],
+              // "za >= ge and lt < za" holds exactly when the peer's first arg-max is a.
+              float vv[V];
+              SegOps<T>::unpack(u_a == 0 ? raw[0] : raw[kSegPerThread - 1], vv);
+              float pre = -INFINITY;
+#pragma unroll
+              for (int i = 0; i < V; ++i) {
+                const int c = seg_a * V - g.head + i;
+                if (c < a_own) pre = fmaxf(pre, vv[i]);
+                if (c == a_own) za[j] = vv[i];
+              }
+              lt[j] = SegOps<T>::mmax(lt[j], SegOps<T>::from_scalar(pre));
+            }
             __syncwarp();
             if (lane == 0) mbar_arrive(&ctrl->ring_empty[st]);
             if (++st == n_stage) { st = 0; st_phase ^= 1u; }
@@ -831,6 +864,13 @@ rows_tma_kernel(const __grid_constant__ KArgs a, const TmaCfg cfg) {
               const float2 e = exp_shift2<T>(z2[u][i], m, l2e2, nml2);
               g2[i] = __ffma2_rn(e, cp2, __ffma2_rn(sd2[u][i], cd2, ncq2));
               if constexpr (!PW) dist2 = __ffma2_rn(sd2[u][i], sd2[u][i], dist2);
+            }
+            if (((spec_y >> k) & 1u) && u == u_y) {  // the label column: q_y carries the extra 1 - eps
+#pragma unroll
+              for (int i = 0; i < H; ++i) {
+                if (2 * i == pos_y) g2[i].x -= cy;
+                if (2 * i + 1 == pos_y) g2[i].y -= cy;
+              }
             }
             *reinterpret_cast<uint4*>(g_img + off + u * (kConsumers * 16)) = SegOps<T>::pack2(g2);
           }
