@@ -22,6 +22,7 @@ __global__ void __launch_bounds__(1024) prep_kernel(WsHeader* hdr, int64_t* part
   __shared__ long long sh[2][32];
   __shared__ int sh_bad;
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  release_dependent_grid();  // the main kernel may start its set-up now; it waits for this grid before reading the workspace
   if (tid == 0) sh_bad = 0;
   __syncthreads();
   long long valid = 0, masked = 0;

@@ -5,6 +5,8 @@
 #include <cuda_runtime.h>
 #include <stdint.h>
 
+#include <utility>
+
 #include "../../include/codistill.h"
 
 namespace codistill {
@@ -66,6 +68,30 @@ struct KArgs {
   int fused_finalize;          // last CTA reduces losses and counters
   float alpha, temperature, eps;
 };
+
+// ------------------------------------------------------------------ programmatic dependent launch
+// The main kernels are launched with programmatic stream serialisation: their CTAs may start while
+// the prep kernel of the same call still runs, so that launch latency and set-up overlap with it.
+// Nothing the prep kernel writes (workspace header, partial counts) may be touched before
+// wait_for_prior_grid() returns; it returns once the preceding grid has finished and its writes are visible.
+__device__ __forceinline__ void wait_for_prior_grid() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+__device__ __forceinline__ void release_dependent_grid() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+
+// Launches `kernel` so that it may overlap the tail of the kernel before it in the stream.
+template <typename... KP, typename... Args>
+inline cudaError_t launch_overlapped(void (*kernel)(KP...), dim3 grid, dim3 block, size_t smem, cudaStream_t stream, Args&&... args) {
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = grid;
+  cfg.blockDim = block;
+  cfg.dynamicSmemBytes = smem;
+  cfg.stream = stream;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = 1;
+  return cudaLaunchKernelEx(&cfg, kernel, std::forward<Args>(args)...);
+}
 
 // ------------------------------------------------------------------ element conversion
 template <typename T> struct Elem;

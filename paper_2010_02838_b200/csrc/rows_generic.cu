@@ -269,6 +269,7 @@ rows_generic_kernel(const __grid_constant__ KArgs a) {
   __shared__ double sh_final[32];
   __shared__ int sh_flag;
 
+  wait_for_prior_grid();
   float w = 1.f;
   if (a.reduction == CODISTILL_REDUCE_MEAN_VALID) {
     const int64_t nv = total_valid(a);
@@ -301,7 +302,8 @@ cudaError_t launch_generic(const KArgs& a, int dtype, bool warp_regime, bool vec
     threads = kBlockRegimeThreads;
     grid = rows < (int64_t)num_sms * 4 ? rows : (int64_t)num_sms * 4;
   }
-#define CODISTILL_LAUNCH(T, V, G) rows_generic_kernel<T, V, G><<<(unsigned)grid, threads, 0, stream>>>(a)
+  cudaError_t err = cudaSuccess;
+#define CODISTILL_LAUNCH(T, V, G) err = launch_overlapped(rows_generic_kernel<T, V, G>, dim3((unsigned)grid), dim3(threads), 0, stream, a)
   if (dtype == CODISTILL_F32) {
     if (warp_regime) { if (vec) CODISTILL_LAUNCH(float, 4, 32); else CODISTILL_LAUNCH(float, 1, 32); }
     else { if (vec) CODISTILL_LAUNCH(float, 4, kBlockRegimeThreads); else CODISTILL_LAUNCH(float, 1, kBlockRegimeThreads); }
@@ -310,7 +312,7 @@ cudaError_t launch_generic(const KArgs& a, int dtype, bool warp_regime, bool vec
     else { if (vec) CODISTILL_LAUNCH(__nv_bfloat16, 8, kBlockRegimeThreads); else CODISTILL_LAUNCH(__nv_bfloat16, 1, kBlockRegimeThreads); }
   }
 #undef CODISTILL_LAUNCH
-  return cudaGetLastError();
+  return err != cudaSuccess ? err : cudaGetLastError();
 }
 
 }  // namespace codistill

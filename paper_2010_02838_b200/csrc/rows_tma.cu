@@ -451,6 +451,7 @@ rows_tma_kernel(const __grid_constant__ KArgs a, const TmaCfg cfg) {
   char* zero_region = reinterpret_cast<char*>(smem_raw) + (kCtrlBytes - kZeroBytes);
   for (int i = threadIdx.x * 16; i < kZeroBytes; i += blockDim.x * 16) *reinterpret_cast<uint4*>(zero_region + i) = make_uint4(0u, 0u, 0u, 0u);
   asm volatile("fence.proxy.async.shared::cta;" ::: "memory");  // the zeros are read by bulk copies later
+  wait_for_prior_grid();  // from here on the workspace header and the valid-row counts are read
   __syncthreads();
 
   if (warp == 0) {
@@ -1083,8 +1084,8 @@ template <typename T, int P, bool PW, int NCW>
 static cudaError_t launch_one(const KArgs& a, const TmaCfg& c, int grid, cudaStream_t stream) {
   cudaError_t e = cudaFuncSetAttribute(rows_tma_kernel<T, P, PW, NCW>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)c.smem_bytes);
   if (e != cudaSuccess) return e;
-  rows_tma_kernel<T, P, PW, NCW><<<grid, NCW * 32 + kProducerThreads, c.smem_bytes, stream>>>(a, c);
-  return cudaGetLastError();
+  e = launch_overlapped(rows_tma_kernel<T, P, PW, NCW>, dim3(grid), dim3(NCW * 32 + kProducerThreads), c.smem_bytes, stream, a, c);
+  return e != cudaSuccess ? e : cudaGetLastError();
 }
 
 template <typename T, int NCW>
