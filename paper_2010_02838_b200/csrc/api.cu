@@ -1,6 +1,7 @@
 // Host side of the C ABI declared in include/codistill.h: argument validation, workspace
 // layout, regime dispatch, the prep / finalize kernels and the host-buffer pipeline.
 #include <math.h>
+#include <stdlib.h>
 #include <string.h>
 
 #include "common.cuh"
@@ -11,7 +12,10 @@ namespace codistill {
 
 cudaError_t launch_generic(const KArgs& a, int dtype, bool warp_regime, bool vec, int num_sms, cudaStream_t stream);
 bool tma_supported(const KArgs& a, int dtype, int smem_optin);
+int tma_ctas_per_sm(const KArgs& a, int dtype, int smem_optin);
 cudaError_t launch_tma(const KArgs& a, int dtype, int num_sms, int smem_optin, cudaStream_t stream);
+bool stream_supported(const KArgs& a, int dtype);
+cudaError_t launch_stream(const KArgs& a, int dtype, int num_sms, cudaStream_t stream);
 
 // ------------------------------------------------------------------ prep and finalize kernels
 // Zeroes the workspace header and counts valid / masked rows (one partial pair per block, summed
@@ -111,12 +115,26 @@ static int validate(const codistill_params_t* p, bool host_pointers) {
   return CODISTILL_OK;
 }
 
-enum Regime { kRegimeWarp = 0, kRegimeBlock = 1, kRegimeTma = 2 };
+enum Regime { kRegimeWarp = 0, kRegimeBlock = 1, kRegimeTma = 2, kRegimeStream = 3 };
 
+// Long rows with the MSE distance have two kernels: "tma" (own row staged in shared memory by bulk
+// copies) and "stream" (direct loads, own row re-read through L2).  The staged kernel is the faster
+// one while two of its CTAs fit an SM (rows up to 64 KiB); beyond that, and for rows it cannot hold
+// at all, the direct-load kernel is.  The environment variable CODISTILL_REGIME = stream | tma |
+// block overrides the default choice where the named kernel supports the call (for measurements;
+// results are the same within rounding).
 static Regime pick_regime(const KArgs& a, int dtype, int smem_optin) {
-  if (tma_supported(a, dtype, smem_optin)) return kRegimeTma;
   const int64_t row_bytes = a.classes * (dtype == CODISTILL_F32 ? 4 : 2);
-  return row_bytes <= 8192 ? kRegimeWarp : kRegimeBlock;
+  const Regime generic = row_bytes <= 8192 ? kRegimeWarp : kRegimeBlock;
+  const bool can_tma = tma_supported(a, dtype, smem_optin), can_stream = stream_supported(a, dtype);
+  if (const char* want = getenv("CODISTILL_REGIME")) {
+    if (strcmp(want, "tma") == 0 && can_tma) return kRegimeTma;
+    if (strcmp(want, "stream") == 0 && can_stream) return kRegimeStream;
+    if (strcmp(want, "block") == 0) return generic;
+  }
+  if (can_tma && (!can_stream || tma_ctas_per_sm(a, dtype, smem_optin) >= 2)) return kRegimeTma;
+  if (can_stream) return kRegimeStream;
+  return generic;
 }
 
 static bool rows_vectorizable(const KArgs& a, int dtype) {
@@ -175,6 +193,7 @@ static cudaError_t launch_prep(const KArgs& a, cudaStream_t stream) {
 static cudaError_t launch_main(const KArgs& a, int dtype, const DeviceInfo& di, cudaStream_t stream) {
   const Regime reg = pick_regime(a, dtype, di.smem_optin);
   if (reg == kRegimeTma) return launch_tma(a, dtype, di.num_sms, di.smem_optin, stream);
+  if (reg == kRegimeStream) return launch_stream(a, dtype, di.num_sms, stream);
   return launch_generic(a, dtype, reg == kRegimeWarp, rows_vectorizable(a, dtype), di.num_sms, stream);
 }
 
@@ -428,6 +447,7 @@ const char* codistill_kernel_regime(int n, int64_t rows, int64_t classes, int64_
   switch (pick_regime(a, dtype, di.smem_optin)) {
     case kRegimeWarp: return "warp";
     case kRegimeBlock: return "block";
+    case kRegimeStream: return "stream";
     default: return "tma";
   }
 }

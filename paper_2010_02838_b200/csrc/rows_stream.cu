@@ -1,0 +1,461 @@
+// Streaming kernel for long rows ("stream" regime), MSE-on-logits distance.
+//
+// One 256-thread CTA works on one row at a time; three CTAs are resident per SM and draw rows
+// from a global counter.  Nothing is staged in shared memory.  Every thread reads its 16-byte
+// segments of the row straight from global memory, several loads in flight per thread:
+//   pass A  the own row once: online softmax (running maximum with its first segment, sum exp,
+//           sum z), then one block reduction gives the row statistics;
+//   pass B  the own row again, together with the n-1 peer rows: differences, squared distance,
+//           what the arg-max agreement needs, the gradient, written with 16-byte stores.
+// The second read of the own row comes a few microseconds after the first and is served by the
+// L2 cache, so that HBM sees every logit once and the gradient once, as in the staged kernel.
+// With no shared-memory row buffer the row length is unbounded: this kernel serves the rows that are
+// too long for the staged kernel (vocabularies beyond about 90 K bf16 classes).
+//
+// Rows need not be 16-byte aligned: a thread works on the segments of the row image (the aligned
+// byte range that holds the row) that lie wholly inside the row; the ragged first / last segments
+// of an unaligned row are done element by element by two designated threads.
+#include <type_traits>
+
+#include "common.cuh"
+#include "seg_math.cuh"
+
+namespace codistill {
+
+#ifndef STREAM_THREADS
+#define STREAM_THREADS 256
+#define STREAM_CTAS 3
+#define STREAM_BATCH_A 4
+#define STREAM_BATCH_B 2
+#endif
+constexpr int kStreamThreads = STREAM_THREADS;
+constexpr int kStreamCtasPerSm = STREAM_CTAS;
+constexpr int kStreamWarps = kStreamThreads / 32;
+constexpr int kStreamMaxPeers = 7;
+constexpr int kBatchA = STREAM_BATCH_A;   // segments per thread in flight in pass A
+constexpr int kBatchB = STREAM_BATCH_B;   // own segments per thread in flight in pass B (plus as many per peer)
+
+struct StreamShared {
+  float4 red[2][kStreamWarps];                              // pass-A partials, alternating between rows
+  float endred[2][kStreamWarps * (1 + 3 * kStreamMaxPeers)];  // pass-B partials, alternating between rows
+  long long next_row[2];
+  double fin[32];
+  int last_flag;
+};
+
+// First column of segment `s` of the row image whose value equals m, or INT_MAX; reads single elements.
+template <typename T>
+__device__ __noinline__ int first_equal_global(const T* __restrict__ z_row, int s, int head, int64_t C, float m) {
+  constexpr int V = SegOps<T>::V;
+  int first = 0x7fffffff;
+#pragma unroll
+  for (int i = V - 1; i >= 0; --i) {
+    const int64_t c = (int64_t)s * V - head + i;
+    if (c >= 0 && c < C && Elem<T>::to_f32(z_row[c]) == m) first = (int)c;
+  }
+  return first;
+}
+
+template <typename T, int P, bool PW>
+__global__ void __launch_bounds__(kStreamThreads, kStreamCtasPerSm) rows_stream_kernel(const __grid_constant__ KArgs a) {
+  constexpr int V = SegOps<T>::V;
+  constexpr int H = SegOps<T>::H;
+  constexpr int PD = P > 0 ? P : 1;
+  constexpr int ES = (int)sizeof(T);
+  constexpr int NT = kStreamThreads;
+  __shared__ StreamShared sh;
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  const int64_t C = a.classes;
+  const bool with_term = (P >= 1 && a.alpha != 0.f);
+  const bool stream_peers = (P >= 1) && (with_term || a.want_flags);
+
+  wait_for_prior_grid();  // from here on the workspace header and the valid-row counts are read
+  float w = 1.f;
+  if (a.reduction == CODISTILL_REDUCE_MEAN_VALID) {
+    const int64_t nv = total_valid(a);
+    w = 1.f / (float)(nv > 1 ? nv : 1);
+  }
+  const float inv_P = P >= 1 ? 1.f / (float)P : 0.f;
+  const float inv_C = 1.f / (float)C;
+  const float2 l2e2 = make_float2(kLog2e, kLog2e);
+  const float2 neg1 = make_float2(-1.f, -1.f);
+
+  if (tid == 0) sh.next_row[0] = a.row_begin + (long long)atomicAdd(&a.hdr->next_row, 1u);
+  __syncthreads();
+  int v = 0;  // valid rows done by this CTA
+  for (int it = 0;; ++it) {
+    const long long r = sh.next_row[it & 1];
+    if (r >= a.row_end) break;
+    if (tid == 0) sh.next_row[(it + 1) & 1] = a.row_begin + (long long)atomicAdd(&a.hdr->next_row, 1u);
+    const int64_t lr = r - a.row_begin;
+    const RowGeom g = row_geom<T>(lr, a.row_stride, C);
+    const int64_t row_off = lr * a.row_stride;  // in elements
+    const T* __restrict__ z_row = reinterpret_cast<const T*>(a.own) + row_off;
+    T* __restrict__ g_row = a.grad ? reinterpret_cast<T*>(a.grad) + row_off : nullptr;
+    const uint4* __restrict__ z_img = reinterpret_cast<const uint4*>(z_row - g.head);
+    uint4* __restrict__ g_img = g_row ? reinterpret_cast<uint4*>(g_row - g.head) : nullptr;
+    const int n_int = g.seg_hi > g.seg_lo ? g.seg_hi - g.seg_lo : 0;    // segments wholly inside the row
+    const int cnt = n_int > tid ? (n_int - tid + NT - 1) / NT : 0;     // of which this thread has cnt: seg_lo + tid + NT * i
+    const int s0 = g.seg_lo + tid;
+    // ragged segments: thread 0 takes the first, thread 32 the last
+    const bool edge_head = (tid == 0) && g.seg_lo > 0;
+    const bool edge_tail = (tid == 32 % NT) && g.seg_hi < g.n_seg && (g.n_seg > 1 || g.seg_lo == 0);
+    const int y = a.labels[r];
+    const bool valid = (a.mask == nullptr || a.mask[r] != 0) && y >= 0 && (int64_t)y < C;
+
+    if (!valid) {  // masked row: zero gradient, no loss, no counts; nothing is read
+      if (g_img) {
+        for (int i = 0; i < cnt; ++i) g_img[s0 + i * NT] = make_uint4(0u, 0u, 0u, 0u);
+        if (edge_head || edge_tail) {
+          const int s = edge_head ? 0 : g.n_seg - 1;
+#pragma unroll
+          for (int i = 0; i < V; ++i) {
+            const int64_t c = (int64_t)s * V - g.head + i;
+            if (c >= 0 && c < C) g_row[c] = Elem<T>::from_f32(0.f);
+          }
+        }
+      }
+      if (tid == 0) { a.row_loss[r] = 0.f; a.row_flags[r] = 0u; }
+      __syncthreads();  // orders the row-id hand-over
+      continue;
+    }
+    const int par = v & 1;
+
+    // ================= pass A: own-row statistics
+    float best = -3.0e38f;  // finite, so that the first rescale is exp2(-huge) = 0 and never NaN
+    int best_seg = 0x7fffffff;
+    float2 s2[H], zs2[H];
+#pragma unroll
+    for (int i = 0; i < H; ++i) { s2[i] = make_float2(0.f, 0.f); zs2[i] = make_float2(0.f, 0.f); }
+    float s_edge = 0.f, z_edge = 0.f;
+    auto sweep_batch = [&](auto nb, int i0) {
+      constexpr int B = decltype(nb)::value;
+      uint4 rw[B];
+#pragma unroll
+      for (int u = 0; u < B; ++u) rw[u] = z_img[s0 + (i0 + u) * NT];
+      const float old_best = best;
+#pragma unroll
+      for (int u = 0; u < B; ++u) {
+        const float fm = SegOps<T>::to_float(SegOps<T>::fold(rw[u]));
+        if (fm > best) { best = fm; best_seg = s0 + (i0 + u) * NT; }
+      }
+      const float sc = rescale_exp2<T>((old_best - best) * kLog2e);
+      const float2 sc2 = make_float2(sc, sc);
+      const float2 nmk = make_float2(-best * kLog2e, -best * kLog2e);
+      s_edge *= sc;
+#pragma unroll
+      for (int i = 0; i < H; ++i) s2[i] = __fmul2_rn(s2[i], sc2);
+#pragma unroll
+      for (int u = 0; u < B; ++u) {
+        float2 z2[H];
+        SegOps<T>::unpack2(rw[u], z2);
+#pragma unroll
+        for (int i = 0; i < H; ++i) {
+          s2[i] = __fadd2_rn(s2[i], exp_shift2<T>(z2[i], best, l2e2, nmk));
+          zs2[i] = __fadd2_rn(zs2[i], z2[i]);
+        }
+      }
+    };
+    {
+      int i = 0;
+      for (; i + kBatchA <= cnt; i += kBatchA) sweep_batch(std::integral_constant<int, kBatchA>{}, i);
+      for (; i < cnt; ++i) sweep_batch(std::integral_constant<int, 1>{}, i);
+    }
+    if (edge_head || edge_tail) {  // ragged segment, element by element
+      const int s = edge_head ? 0 : g.n_seg - 1;
+      float zv[V];
+      float fm = -3.0e38f;
+#pragma unroll
+      for (int i = 0; i < V; ++i) {
+        const int64_t c = (int64_t)s * V - g.head + i;
+        zv[i] = (c >= 0 && c < C) ? Elem<T>::to_f32(z_row[c]) : -INFINITY;
+        fm = fmaxf(fm, zv[i]);
+      }
+      const float old_best = best;
+      if (fm > best || (fm == best && s < best_seg)) { best = fm; best_seg = s; }
+      const float sc = rescale_exp2<T>((old_best - best) * kLog2e);
+      const float2 sc2 = make_float2(sc, sc);
+      const float2 nmk = make_float2(-best * kLog2e, -best * kLog2e);
+      s_edge *= sc;
+#pragma unroll
+      for (int i = 0; i < H; ++i) s2[i] = __fmul2_rn(s2[i], sc2);
+#pragma unroll
+      for (int i = 0; i < V; ++i) {
+        if (zv[i] != -INFINITY) {
+          s_edge += exp_shift2<T>(make_float2(zv[i], zv[i]), best, l2e2, nmk).x;
+          z_edge += zv[i];
+        }
+      }
+    }
+    float s_t = s_edge, z_t = z_edge;
+#pragma unroll
+    for (int i = 0; i < H; ++i) { s_t += s2[i].x + s2[i].y; z_t += zs2[i].x + zs2[i].y; }
+    // block reduction in one round: maximum with its first segment, then the sums rescaled to it
+    float m;
+    int m_seg;
+    float S = 0.f, sum_z = 0.f;
+    {
+      const unsigned key = float_order_key(best + 0.f);  // -0 is folded onto +0: they tie
+      const unsigned key_w = __reduce_max_sync(0xffffffffu, key);
+      const int seg_w = (int)__reduce_min_sync(0xffffffffu, key == key_w ? (unsigned)best_seg : 0x7fffffffu);
+      const float m_w = float_from_order_key(key_w);
+      const float sw = warp_sum(s_t * rescale_exp2<T>((best - m_w) * kLog2e));
+      const float zw = warp_sum(z_t);
+      if (lane == 0) sh.red[par][warp] = make_float4(m_w, __int_as_float(seg_w), sw, zw);
+      __syncthreads();
+      float4 part[kStreamWarps];
+#pragma unroll
+      for (int wv = 0; wv < kStreamWarps; ++wv) part[wv] = sh.red[par][wv];
+      m = part[0].x;
+      m_seg = __float_as_int(part[0].y);
+#pragma unroll
+      for (int wv = 1; wv < kStreamWarps; ++wv) argmax_combine(m, m_seg, part[wv].x, __float_as_int(part[wv].y));
+#pragma unroll
+      for (int wv = 0; wv < kStreamWarps; ++wv) {
+        S += part[wv].z * rescale_exp2<T>((part[wv].x - m) * kLog2e);
+        sum_z += part[wv].w;
+      }
+    }
+    if (m_seg >= g.n_seg) m_seg = 0;  // NaN rows: keep the reads below inside the row
+    const int a_own = first_equal_global<T>(z_row, m_seg, g.head, C, m);
+    const int seg_a = a.want_flags ? m_seg : -1;
+    const float zy = Elem<T>::to_f32(z_row[y]);
+
+    // ================= pass B: peers, distance, gradient
+    const float2 nml2 = make_float2(-m * kLog2e, -m * kLog2e);
+    const float cp = w * __frcp_rn(S);                                          // e_c -> w * p_c
+    const float cd = with_term ? w * a.alpha * (2.f * inv_C) * inv_P : 0.f;     // sum_j d -> w * alpha * dD
+    const float cq = w * a.eps * inv_C;
+    const float cy = w * (1.f - a.eps);
+    const float2 cp2 = make_float2(cp, cp), cd2 = make_float2(cd, cd), ncq2 = make_float2(-cq, -cq);
+    const int seg_y = (g.head + y) / V, pos_y = (g.head + y) % V;
+    float2 dist2 = make_float2(0.f, 0.f), dist2b = make_float2(0.f, 0.f);
+    typename SegOps<T>::macc lt[PD], ge[PD];
+    float za[PD];
+#pragma unroll
+    for (int j = 0; j < PD; ++j) { lt[j] = SegOps<T>::neg_inf(); ge[j] = SegOps<T>::neg_inf(); za[j] = -INFINITY; }
+    const uint4* p_img[PD];
+#pragma unroll
+    for (int j = 0; j < PD; ++j)
+      p_img[j] = P > 0 ? reinterpret_cast<const uint4*>(reinterpret_cast<const T*>(a.peers[j]) + row_off - g.head) : nullptr;
+
+    auto grad_batch = [&](auto nb, int i0) {
+      constexpr int B = decltype(nb)::value;
+      uint4 zr[B];
+#pragma unroll
+      for (int u = 0; u < B; ++u) zr[u] = z_img[s0 + (i0 + u) * NT];
+      float2 z2[B][H], sd2[B][H];
+#pragma unroll
+      for (int u = 0; u < B; ++u) {
+#pragma unroll
+        for (int i = 0; i < H; ++i) sd2[u][i] = make_float2(0.f, 0.f);
+      }
+      if (stream_peers) {
+#pragma unroll
+        for (int u = 0; u < B; ++u) SegOps<T>::unpack2(zr[u], z2[u]);
+        // the peers in groups of at most four, so that the loads in flight fit the register budget
+        constexpr int PG = PD < 4 ? PD : 4;
+#pragma unroll
+        for (int j0 = 0; j0 < P; j0 += PG) {
+        uint4 pr[PG][B];
+#pragma unroll
+        for (int jj = 0; jj < PG; ++jj) {
+          if (j0 + jj < P) {
+#pragma unroll
+            for (int u = 0; u < B; ++u) pr[jj][u] = p_img[j0 + jj][s0 + (i0 + u) * NT];
+          }
+        }
+#pragma unroll
+        for (int jj = 0; jj < PG; ++jj) {
+          const int j = j0 + jj;
+          if (j >= P) break;
+#pragma unroll
+          for (int u = 0; u < B; ++u) {
+            const int s = s0 + (i0 + u) * NT;
+            float2 v2[H];
+            SegOps<T>::unpack2(pr[jj][u], v2);
+#pragma unroll
+            for (int i = 0; i < H; ++i) {
+              const float2 d = __ffma2_rn(v2[i], neg1, z2[u][i]);
+              if (P == 1 || j == 0) sd2[u][i] = d; else sd2[u][i] = __fadd2_rn(sd2[u][i], d);
+              if constexpr (PW) { if (i & 1) dist2b = __ffma2_rn(d, d, dist2b); else dist2 = __ffma2_rn(d, d, dist2); }
+            }
+            const typename SegOps<T>::macc f = SegOps<T>::fold(pr[jj][u]);
+            const bool before = s < seg_a;
+            lt[j] = before ? SegOps<T>::mmax(lt[j], f) : lt[j];
+            ge[j] = before ? ge[j] : SegOps<T>::mmax(ge[j], f);
+            if (s == seg_a) {
+              // The segment of the own arg-max column a went to ge[] as a whole.  The peer's value at a and
+              // the largest value before a inside the segment settle the rest: with them in za[] and lt[],
+              // "za >= ge and lt < za" holds exactly when the peer's first arg-max is a.
+              float vv[V];
+              SegOps<T>::unpack(pr[jj][u], vv);
+              float pre = -INFINITY;
+#pragma unroll
+              for (int i = 0; i < V; ++i) {
+                const int c = seg_a * V - g.head + i;
+                if (c < a_own) pre = fmaxf(pre, vv[i]);
+                if (c == a_own) za[j] = vv[i];
+              }
+              lt[j] = SegOps<T>::mmax(lt[j], SegOps<T>::from_scalar(pre));
+            }
+          }
+        }
+        }
+      } else {
+#pragma unroll
+        for (int u = 0; u < B; ++u) SegOps<T>::unpack2(zr[u], z2[u]);
+      }
+#pragma unroll
+      for (int u = 0; u < B; ++u) {
+        const int s = s0 + (i0 + u) * NT;
+        float2 g2[H];
+#pragma unroll
+        for (int i = 0; i < H; ++i) {
+          const float2 e = exp_shift2<T>(z2[u][i], m, l2e2, nml2);
+          g2[i] = __ffma2_rn(e, cp2, __ffma2_rn(sd2[u][i], cd2, ncq2));
+          if constexpr (!PW) dist2 = __ffma2_rn(sd2[u][i], sd2[u][i], dist2);  // (sum_j d)^2, scaled by 1/P^2 below
+        }
+        if (s == seg_y) {  // the label column: q_y carries the extra 1 - eps
+#pragma unroll
+          for (int i = 0; i < H; ++i) {
+            if (2 * i == pos_y) g2[i].x -= cy;
+            if (2 * i + 1 == pos_y) g2[i].y -= cy;
+          }
+        }
+        if (g_img) g_img[s] = SegOps<T>::pack2(g2);
+      }
+    };
+    {
+      int i = 0;
+      constexpr int BB = P >= 3 ? 1 : kBatchB;
+      for (; i + BB <= cnt; i += BB) grad_batch(std::integral_constant<int, BB>{}, i);
+      for (; i < cnt; ++i) grad_batch(std::integral_constant<int, 1>{}, i);
+    }
+    float dist_edge = 0.f;
+    if (edge_head || edge_tail) {  // ragged segment, element by element
+      const int s = edge_head ? 0 : g.n_seg - 1;
+#pragma unroll
+      for (int i = 0; i < V; ++i) {
+        const int64_t c = (int64_t)s * V - g.head + i;
+        if (c < 0 || c >= C) continue;
+        const float z = Elem<T>::to_f32(z_row[c]);
+        float sd = 0.f;
+        if (stream_peers) {
+#pragma unroll
+          for (int j = 0; j < P; ++j) {
+            const float pv = Elem<T>::to_f32(reinterpret_cast<const T*>(a.peers[j])[row_off + c]);
+            const float d = z - pv;
+            sd += d;
+            if constexpr (PW) dist_edge = fmaf(d, d, dist_edge);
+            if (a.want_flags) {
+              if (c < a_own) lt[j] = SegOps<T>::mmax(lt[j], SegOps<T>::from_scalar(pv));
+              else if (c > a_own) ge[j] = SegOps<T>::mmax(ge[j], SegOps<T>::from_scalar(pv));
+              else za[j] = pv;
+            }
+          }
+        }
+        if constexpr (!PW) dist_edge = fmaf(sd, sd, dist_edge);
+        const float e = exp_shift2<T>(make_float2(z, z), m, l2e2, nml2).x;
+        float gv = fmaf(e, cp, fmaf(sd, cd, -cq));
+        if (c == (int64_t)y) gv -= cy;
+        if (g_row) g_row[c] = Elem<T>::from_f32(gv);
+      }
+    }
+
+    // ================= row results: per-warp partials, then warp 0 finishes the row
+    {
+      float part[1 + 3 * PD];
+      part[0] = warp_sum((dist2.x + dist2.y) + (dist2b.x + dist2b.y) + dist_edge);
+#pragma unroll
+      for (int j = 0; j < PD; ++j) {
+        part[1 + 3 * j] = warp_max_redux(SegOps<T>::to_float(lt[j]));
+        part[2 + 3 * j] = warp_max_redux(SegOps<T>::to_float(ge[j]));
+        part[3 + 3 * j] = warp_max_redux(za[j]);
+      }
+      if (lane == 0) {
+#pragma unroll
+        for (int i = 0; i < 1 + 3 * PD; ++i) sh.endred[par][i * kStreamWarps + warp] = part[i];
+      }
+      __syncthreads();
+      if (warp == 0) {
+        const float* er = sh.endred[par];
+        const float dsum = warp_sum(lane < kStreamWarps ? er[lane] : 0.f);
+        uint32_t flags = 0u;
+        if (a.want_flags) {
+          flags = (a_own == y) ? 1u : 0u;
+#pragma unroll
+          for (int j = 0; j < P; ++j) {
+            const float ltv = warp_max_redux(lane < kStreamWarps ? er[(1 + 3 * j) * kStreamWarps + lane] : -INFINITY);
+            const float gev = warp_max_redux(lane < kStreamWarps ? er[(2 + 3 * j) * kStreamWarps + lane] : -INFINITY);
+            const float zav = warp_max_redux(lane < kStreamWarps ? er[(3 + 3 * j) * kStreamWarps + lane] : -INFINITY);
+            if (zav >= gev && ltv < zav) flags |= (2u << j);
+          }
+        }
+        if (lane == 0) {
+          const float ce = (m + logf(S)) - (1.f - a.eps) * zy - (a.eps * inv_C) * sum_z;
+          float D = 0.f;
+          if (with_term) D = PW ? dsum * inv_P * inv_C : dsum * inv_P * inv_P * inv_C;
+          a.row_loss[r] = with_term ? fmaf(a.alpha, D, ce) : ce;
+          a.row_flags[r] = flags;
+        }
+      }
+    }
+    ++v;
+  }
+
+  // ---------------- all rows of this CTA are written: scheduler reset and final reduction
+  __threadfence();
+  __syncthreads();
+  if (tid == 0) {
+    const unsigned int prev = atomicAdd(&a.hdr->sched_done, 1u);
+    sh.last_flag = (prev == gridDim.x - 1);
+    if (sh.last_flag) { a.hdr->next_row = 0u; a.hdr->sched_done = 0u; __threadfence(); }  // ready for the next launch
+  }
+  __syncthreads();
+  if (a.fused_finalize && sh.last_flag) {
+    __threadfence();
+    finalize_cta(a, sh.fin);
+  }
+}
+
+// ------------------------------------------------------------------ host side
+bool stream_supported(const KArgs& a, int dtype) {
+  const int64_t es = dtype == CODISTILL_F32 ? 4 : 2;
+  if (a.dist != CODISTILL_DIST_MSE_LOGITS) return false;
+  if (!(a.n_peers == 0 || a.n_peers == 1 || a.n_peers == 2 || a.n_peers == 3 || a.n_peers == 7)) return false;
+  if (a.classes * es < 8192 || a.classes > (int64_t)1 << 24) return false;
+  uintptr_t bits = reinterpret_cast<uintptr_t>(a.own) | reinterpret_cast<uintptr_t>(a.grad);
+  for (int j = 0; j < a.n_peers; ++j) bits |= reinterpret_cast<uintptr_t>(a.peers[j]);
+  return (bits & 15u) == 0;
+}
+
+template <typename T, int P, bool PW>
+static cudaError_t stream_launch_one(const KArgs& a, int grid, cudaStream_t stream) {
+  const cudaError_t e = launch_overlapped(rows_stream_kernel<T, P, PW>, dim3(grid), dim3(kStreamThreads), 0, stream, a);
+  return e != cudaSuccess ? e : cudaGetLastError();
+}
+
+template <typename T>
+static cudaError_t stream_launch_peers(const KArgs& a, int grid, cudaStream_t stream) {
+  const bool pw = a.peer_reduce == CODISTILL_PEERS_PAIRWISE_MEAN;  // with one peer both readings coincide
+  switch (a.n_peers) {
+    case 0: return stream_launch_one<T, 0, true>(a, grid, stream);
+    case 1: return stream_launch_one<T, 1, true>(a, grid, stream);
+    case 2: return pw ? stream_launch_one<T, 2, true>(a, grid, stream) : stream_launch_one<T, 2, false>(a, grid, stream);
+    case 3: return pw ? stream_launch_one<T, 3, true>(a, grid, stream) : stream_launch_one<T, 3, false>(a, grid, stream);
+    case 7: return pw ? stream_launch_one<T, 7, true>(a, grid, stream) : stream_launch_one<T, 7, false>(a, grid, stream);
+    default: return cudaErrorNotSupported;
+  }
+}
+
+cudaError_t launch_stream(const KArgs& a, int dtype, int num_sms, cudaStream_t stream) {
+  if (!stream_supported(a, dtype)) return cudaErrorNotSupported;
+  const int64_t rows = a.row_end - a.row_begin;
+  if (rows <= 0) return cudaSuccess;
+  const int64_t slots = (int64_t)num_sms * kStreamCtasPerSm;
+  const int grid = (int)(rows < slots ? rows : slots);
+  return dtype == CODISTILL_F32 ? stream_launch_peers<float>(a, grid, stream) : stream_launch_peers<__nv_bfloat16>(a, grid, stream);
+}
+
+}  // namespace codistill

@@ -24,6 +24,7 @@
 // that are only partly inside the row ("edge" segments) take a masked slow path.  Every valid row
 // uses the same number of pieces (some possibly empty), so that barrier phases advance uniformly.
 #include "common.cuh"
+#include "seg_math.cuh"
 
 namespace codistill {
 
@@ -121,7 +122,11 @@ __device__ __noinline__ void wait_slow(uint64_t* bar, uint32_t parity, Ctrl* ctr
   volatile int* abort_flag = &ctrl->abort_flag;
   uint32_t polls = 0;
   unsigned long long t0 = 0;
+  // The producer warps wait most of the time and have slack (ring stages, row pieces ahead): they
+  // back off between polls, so that their polling does not take issue slots from the consumers.
+  const bool producer = threadIdx.x < kProducerThreads;
   while (!mbar_try_wait(bar, parity)) {
+    if (producer) __nanosleep(128);
     if ((++polls & 0x3FFu) == 0) {
       if (*abort_flag) return;
       const unsigned long long now = global_timer_ns();
@@ -138,127 +143,6 @@ __device__ __noinline__ void wait_slow(uint64_t* bar, uint32_t parity, Ctrl* ctr
 __device__ __forceinline__ void wait_bounded(uint64_t* bar, uint32_t parity, Ctrl* ctrl, WsHeader* hdr) {
   if (mbar_try_wait(bar, parity)) return;
   wait_slow(bar, parity, ctrl, hdr);
-}
-
-// ------------------------------------------------------------------ 16-byte segments
-template <typename T> struct SegOps;
-template <> struct SegOps<float> {
-  static constexpr int V = 4;   // elements per segment
-  static constexpr int H = 2;   // float2 pairs per segment
-  using macc = float;           // running-maximum accumulator
-  __device__ static void unpack(const uint4& r, float (&o)[4]) {
-    o[0] = __uint_as_float(r.x); o[1] = __uint_as_float(r.y); o[2] = __uint_as_float(r.z); o[3] = __uint_as_float(r.w);
-  }
-  __device__ static void unpack2(const uint4& r, float2 (&o)[2]) {
-    o[0] = make_float2(__uint_as_float(r.x), __uint_as_float(r.y));
-    o[1] = make_float2(__uint_as_float(r.z), __uint_as_float(r.w));
-  }
-  __device__ static uint4 pack2(const float2 (&v)[2]) {
-    return make_uint4(__float_as_uint(v[0].x), __float_as_uint(v[0].y), __float_as_uint(v[1].x), __float_as_uint(v[1].y));
-  }
-  __device__ static macc neg_inf() { return -INFINITY; }
-  __device__ static macc fold(const uint4& r) {
-    return fmaxf(fmaxf(__uint_as_float(r.x), __uint_as_float(r.y)), fmaxf(__uint_as_float(r.z), __uint_as_float(r.w)));
-  }
-  __device__ static macc mmax(macc a, macc b) { return fmaxf(a, b); }
-  __device__ static macc from_scalar(float v) { return v; }
-  __device__ static float to_float(macc a) { return a; }
-};
-template <> struct SegOps<__nv_bfloat16> {
-  static constexpr int V = 8;
-  static constexpr int H = 4;
-  using macc = __nv_bfloat162;  // two running maxima (even / odd columns), folded at the end
-  __device__ static void unpack(const uint4& r, float (&o)[8]) {
-    const uint32_t w[4] = {r.x, r.y, r.z, r.w};
-#pragma unroll
-    for (int i = 0; i < 4; ++i) {
-      o[2 * i] = __uint_as_float(w[i] << 16);
-      o[2 * i + 1] = __uint_as_float(w[i] & 0xFFFF0000u);
-    }
-  }
-  __device__ static void unpack2(const uint4& r, float2 (&o)[4]) {
-    const uint32_t w[4] = {r.x, r.y, r.z, r.w};
-#pragma unroll
-    for (int i = 0; i < 4; ++i) o[i] = make_float2(__uint_as_float(w[i] << 16), __uint_as_float(w[i] & 0xFFFF0000u));
-  }
-  __device__ static uint4 pack2(const float2 (&v)[4]) {
-    uint32_t w[4];
-#pragma unroll
-    for (int i = 0; i < 4; ++i) {
-      const __nv_bfloat162 p = __floats2bfloat162_rn(v[i].x, v[i].y);
-      w[i] = *reinterpret_cast<const uint32_t*>(&p);
-    }
-    return make_uint4(w[0], w[1], w[2], w[3]);
-  }
-  __device__ static macc neg_inf() { return __floats2bfloat162_rn(-INFINITY, -INFINITY); }
-  __device__ static macc fold(const uint4& r) {
-    const __nv_bfloat162 a = __hmax2(*reinterpret_cast<const __nv_bfloat162*>(&r.x), *reinterpret_cast<const __nv_bfloat162*>(&r.y));
-    const __nv_bfloat162 b = __hmax2(*reinterpret_cast<const __nv_bfloat162*>(&r.z), *reinterpret_cast<const __nv_bfloat162*>(&r.w));
-    return __hmax2(a, b);
-  }
-  __device__ static macc mmax(macc a, macc b) { return __hmax2(a, b); }
-  __device__ static macc from_scalar(float v) { return __floats2bfloat162_rn(v, v); }  // v is a bf16 value: exact
-  __device__ static float to_float(macc a) { return fmaxf(__low2float(a), __high2float(a)); }
-};
-
-__device__ __forceinline__ float ex2_approx(float x) {
-  float y;
-  asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
-  return y;
-}
-// exp(z - m) for a pair of columns.  fp32 logits keep full precision (their gradient tolerance is
-// 1e-6 absolute); bf16 logits fold the shift into one packed FMA feeding the hardware exp2.
-template <typename T>
-__device__ __forceinline__ float2 exp_shift2(float2 z, float m, float2 l2e, float2 neg_m_l2e) {
-  if constexpr (sizeof(T) == 4) {
-    return make_float2(expf(z.x - m), expf(z.y - m));
-  } else {
-    const float2 t = __ffma2_rn(z, l2e, neg_m_l2e);
-    return make_float2(ex2_approx(t.x), ex2_approx(t.y));
-  }
-}
-
-// 2^x for the rescaling factors of the online softmax: exact enough for the 1e-6 gradient tolerance of
-// fp32 logits, the bare hardware instruction for bf16 logits.
-template <typename T>
-__device__ __forceinline__ float rescale_exp2(float x) {
-  if constexpr (sizeof(T) == 4) return exp2f(x); else return ex2_approx(x);
-}
-
-// Order-preserving map between floats and unsigned integers (for integer warp reductions).
-__device__ __forceinline__ unsigned float_order_key(float f) {
-  const unsigned u = __float_as_uint(f);
-  return (u & 0x80000000u) ? ~u : (u | 0x80000000u);
-}
-__device__ __forceinline__ float float_from_order_key(unsigned k) {
-  return __uint_as_float((k & 0x80000000u) ? (k & 0x7fffffffu) : ~k);
-}
-
-// Geometry of one row image.
-struct RowGeom {
-  int head;      // elements of the first segment that precede the row
-  int n_seg;     // 16-byte segments of the image
-  int seg_lo;    // first segment that lies wholly inside the row
-  int seg_hi;    // one past the last such segment
-};
-template <typename T>
-__device__ __forceinline__ RowGeom row_geom(int64_t local_row, int64_t row_stride, int64_t classes) {
-  constexpr int V = SegOps<T>::V;
-  RowGeom g;
-  g.head = (int)((local_row * row_stride) & (V - 1));
-  const int64_t end = g.head + classes;  // in elements, from the image start
-  g.n_seg = (int)((end + V - 1) / V);
-  g.seg_lo = g.head ? 1 : 0;
-  g.seg_hi = (end & (V - 1)) ? g.n_seg - 1 : g.n_seg;
-  return g;
-}
-
-// Geometry shared by every row of a call: segments of the longest row image.
-template <typename T>
-__host__ __device__ inline int64_t max_row_segments(int64_t row_stride, int64_t classes) {
-  constexpr int V = 16 / (int)sizeof(T);
-  const int64_t head_max = (row_stride % V == 0) ? 0 : V - 1;
-  return (head_max + classes + V - 1) / V;
 }
 
 // Block reductions among the NCW * 32 consumer threads (one named barrier each).
@@ -606,6 +490,7 @@ rows_tma_kernel(const __grid_constant__ KArgs a, const TmaCfg cfg) {
       w = 1.f / (float)(nv > 1 ? nv : 1);
     }
     const float inv_P = P >= 1 ? 1.f / (float)P : 0.f;
+    const float inv_C = 1.f / (float)C;
     int st = 0;              // ring stage of the next item
     uint32_t st_phase = 0;   // its phase bit
     int v = 0;               // valid rows processed so far
@@ -778,12 +663,13 @@ rows_tma_kernel(const __grid_constant__ KArgs a, const TmaCfg cfg) {
       const int a_own = first_equal<T>(img, m_seg, g.head, C, m);
       const int seg_a = a.want_flags ? m_seg : -1;
       const float zy = Elem<T>::to_f32(reinterpret_cast<const T*>(img)[g.head + y]);
-      const float ce = (m + logf(S)) - (1.f - a.eps) * zy - (a.eps / (float)C) * sum_z;
+      float ce = 0.f;  // task loss of the row: only the thread that publishes it computes it
+      if (red.warp == 0 && lane == 0) ce = (m + logf(S)) - (1.f - a.eps) * zy - (a.eps * inv_C) * sum_z;
 
       // ---------------- stream the peers chunk by chunk, write the gradient, release the own pieces
-      const float cp = w / S;                                                     // e_c -> w * p_c
-      const float cd = with_term ? w * a.alpha * (2.f / (float)C) * inv_P : 0.f;  // sum_j d -> w * alpha * dD
-      const float cq = w * a.eps / (float)C;
+      const float cp = w * __frcp_rn(S);                                          // e_c -> w * p_c
+      const float cd = with_term ? w * a.alpha * (2.f * inv_C) * inv_P : 0.f;     // sum_j d -> w * alpha * dD
+      const float cq = w * a.eps * inv_C;
       const float cy = w * (1.f - a.eps);
       const float2 cp2 = make_float2(cp, cp), cd2 = make_float2(cd, cd), ncq2 = make_float2(-cq, -cq);
       const float2 neg1 = make_float2(-1.f, -1.f);
@@ -1006,9 +892,9 @@ rows_tma_kernel(const __grid_constant__ KArgs a, const TmaCfg cfg) {
         part[0] = warp_sum((dist2.x + dist2.y) + (dist2b.x + dist2b.y));
 #pragma unroll
         for (int j = 0; j < PD; ++j) {
-          part[1 + 3 * j] = warp_max(SegOps<T>::to_float(lt[j]));
-          part[2 + 3 * j] = warp_max(SegOps<T>::to_float(ge[j]));
-          part[3 + 3 * j] = warp_max(za[j]);
+          part[1 + 3 * j] = warp_max_redux(SegOps<T>::to_float(lt[j]));
+          part[2 + 3 * j] = warp_max_redux(SegOps<T>::to_float(ge[j]));
+          part[3 + 3 * j] = warp_max_redux(za[j]);
         }
         if (done >= 2) wait_bounded(&ctrl->end_empty[par], (uint32_t)((done >> 1) - 1) & 1u, ctrl, a.hdr);
         if (lane == 0) {
@@ -1078,6 +964,12 @@ static bool tma_config(const KArgs& a, int dtype, int smem_optin, TmaCfg* out) {
 bool tma_supported(const KArgs& a, int dtype, int smem_optin) {
   TmaCfg c;
   return tma_config(a, dtype, smem_optin, &c);
+}
+
+// CTAs per SM the staged kernel would run with (0: it does not take the call).
+int tma_ctas_per_sm(const KArgs& a, int dtype, int smem_optin) {
+  TmaCfg c;
+  return tma_config(a, dtype, smem_optin, &c) ? c.ctas_per_sm : 0;
 }
 
 template <typename T, int P, bool PW, int NCW>

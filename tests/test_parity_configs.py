@@ -35,7 +35,18 @@ def test_workload_parity(idx, dist, pr, red):
     plan, _, _ = compare(own, peers, labels, mask, alpha=w.alpha, temperature=w.temperature,
                          label_smoothing=w.label_smoothing, dist=dist, peer_reduce=pr, reduction=red)
     if dist == cb.DIST_MSE_LOGITS:   # which kernel served the workload
-        assert plan.regime == {1: "warp", 2: "warp", 3: "warp", 4: "tma", 5: "tma"}[idx]
+        assert plan.regime == {1: "warp", 2: "warp", 3: "warp", 4: "tma", 5: "stream"}[idx]
+
+
+@pytest.mark.parametrize("idx,regime", [(4, "stream"), (5, "tma")])
+@pytest.mark.parametrize("pr,red", list(itertools.product(PEERS, REDS)))
+def test_workload_parity_other_long_row_kernel(monkeypatch, idx, regime, pr, red):
+    """The two largest workloads on the long-row kernel that is not their default."""
+    monkeypatch.setenv("CODISTILL_REGIME", regime)
+    w = workload(idx)
+    own, peers, labels, mask = synth.make_inputs(w)
+    compare(own, peers, labels, mask, alpha=w.alpha, temperature=w.temperature, label_smoothing=w.label_smoothing,
+            dist=cb.DIST_MSE_LOGITS, peer_reduce=pr, reduction=red, expect_regime=regime)
 
 
 @pytest.mark.parametrize("idx", [1, 2, 3])

@@ -25,7 +25,7 @@ def test_full_size_workload(idx):
     d_own, d_peers = to_device(own), [to_device(p) for p in peers]
     plan = cb.Plan(d_own, d_peers, to_device(labels), to_device(mask), alpha=w.alpha, temperature=w.temperature,
                    label_smoothing=w.label_smoothing)
-    assert plan.regime == "tma"
+    assert plan.regime == {4: "tma", 5: "stream"}[idx]      # the launch configuration the benchmark times
     out = plan.run()
     torch.cuda.synchronize()
     assert out.status.item() == 0
