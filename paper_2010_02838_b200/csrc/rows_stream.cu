@@ -1,6 +1,6 @@
 // Streaming kernel for long rows ("stream" regime), MSE-on-logits distance.
 //
-// One 256-thread CTA works on one row at a time; three CTAs are resident per SM and draw rows
+// One CTA of 256 (many peers: 128) threads works on one row at a time; several CTAs are resident per SM and draw rows
 // from a global counter.  Nothing is staged in shared memory.  Every thread reads its 16-byte
 // segments of the row straight from global memory, several loads in flight per thread:
 //   pass A  the own row once: online softmax (running maximum with its first segment, sum exp,
@@ -22,22 +22,19 @@
 
 namespace codistill {
 
-#ifndef STREAM_THREADS
-#define STREAM_THREADS 256
-#define STREAM_CTAS 3
-#define STREAM_BATCH_A 4
-#define STREAM_BATCH_B 2
-#endif
-constexpr int kStreamThreads = STREAM_THREADS;
-constexpr int kStreamCtasPerSm = STREAM_CTAS;
-constexpr int kStreamWarps = kStreamThreads / 32;
+// Launch shape by peer count (measured on B200): up to three peers 256 threads x 3 CTAs per SM
+// (80 registers, two own segments and their peer segments in flight per thread); more peers 128
+// threads x 4 CTAs (128 registers), one own segment and all its peer segments in flight.
+constexpr int kStreamMaxWarps = 8;
 constexpr int kStreamMaxPeers = 7;
-constexpr int kBatchA = STREAM_BATCH_A;   // segments per thread in flight in pass A
-constexpr int kBatchB = STREAM_BATCH_B;   // own segments per thread in flight in pass B (plus as many per peer)
+constexpr int kBatchA = 4;   // segments per thread in flight in pass A
+constexpr int kBatchB = 2;   // own segments per thread in flight in pass B with few peers
+__host__ __device__ constexpr int stream_threads(int peers) { return peers >= 4 ? 128 : 256; }
+__host__ __device__ constexpr int stream_ctas_per_sm(int peers) { return peers >= 4 ? 4 : 3; }
 
 struct StreamShared {
-  float4 red[2][kStreamWarps];                              // pass-A partials, alternating between rows
-  float endred[2][kStreamWarps * (1 + 3 * kStreamMaxPeers)];  // pass-B partials, alternating between rows
+  float4 red[2][kStreamMaxWarps];                              // pass-A partials, alternating between rows
+  float endred[2][kStreamMaxWarps * (1 + 3 * kStreamMaxPeers)];  // pass-B partials, alternating between rows
   long long next_row[2];
   double fin[32];
   int last_flag;
@@ -57,12 +54,13 @@ __device__ __noinline__ int first_equal_global(const T* __restrict__ z_row, int 
 }
 
 template <typename T, int P, bool PW>
-__global__ void __launch_bounds__(kStreamThreads, kStreamCtasPerSm) rows_stream_kernel(const __grid_constant__ KArgs a) {
+__global__ void __launch_bounds__(stream_threads(P), stream_ctas_per_sm(P)) rows_stream_kernel(const __grid_constant__ KArgs a) {
   constexpr int V = SegOps<T>::V;
   constexpr int H = SegOps<T>::H;
   constexpr int PD = P > 0 ? P : 1;
   constexpr int ES = (int)sizeof(T);
-  constexpr int NT = kStreamThreads;
+  constexpr int NT = stream_threads(P);
+  constexpr int kStreamWarps = NT / 32;
   __shared__ StreamShared sh;
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const int64_t C = a.classes;
@@ -253,8 +251,7 @@ __global__ void __launch_bounds__(kStreamThreads, kStreamCtasPerSm) rows_stream_
       if (stream_peers) {
 #pragma unroll
         for (int u = 0; u < B; ++u) SegOps<T>::unpack2(zr[u], z2[u]);
-        // the peers in groups of at most four, so that the loads in flight fit the register budget
-        constexpr int PG = PD < 4 ? PD : 4;
+        constexpr int PG = PD;
 #pragma unroll
         for (int j0 = 0; j0 < P; j0 += PG) {
         uint4 pr[PG][B];
@@ -432,7 +429,7 @@ bool stream_supported(const KArgs& a, int dtype) {
 
 template <typename T, int P, bool PW>
 static cudaError_t stream_launch_one(const KArgs& a, int grid, cudaStream_t stream) {
-  const cudaError_t e = launch_overlapped(rows_stream_kernel<T, P, PW>, dim3(grid), dim3(kStreamThreads), 0, stream, a);
+  const cudaError_t e = launch_overlapped(rows_stream_kernel<T, P, PW>, dim3(grid), dim3(stream_threads(P)), 0, stream, a);
   return e != cudaSuccess ? e : cudaGetLastError();
 }
 
@@ -453,7 +450,7 @@ cudaError_t launch_stream(const KArgs& a, int dtype, int num_sms, cudaStream_t s
   if (!stream_supported(a, dtype)) return cudaErrorNotSupported;
   const int64_t rows = a.row_end - a.row_begin;
   if (rows <= 0) return cudaSuccess;
-  const int64_t slots = (int64_t)num_sms * kStreamCtasPerSm;
+  const int64_t slots = (int64_t)num_sms * stream_ctas_per_sm(a.n_peers);
   const int grid = (int)(rows < slots ? rows : slots);
   return dtype == CODISTILL_F32 ? stream_launch_peers<float>(a, grid, stream) : stream_launch_peers<__nv_bfloat16>(a, grid, stream);
 }
