@@ -118,10 +118,11 @@ def hbm_peak():
     return FALLBACK_HBM_GBS, "fallback (earlier pool measurement)"
 
 
-def kernel_source_hash():
+def kernel_source_hash(files):
+    """Hash of the named kernel sources (the files a stored ncu capture depends on)."""
     h = hashlib.sha256()
     d = os.path.join(ROOT, "paper_2010_02838_b200", "csrc")
-    for f in sorted(os.listdir(d)):
+    for f in sorted(files):
         h.update(open(os.path.join(d, f), "rb").read())
     return h.hexdigest()[:16]
 
@@ -133,7 +134,7 @@ def stored_traffic(workload_idx, dist):
         return None
     try:
         rec = json.load(open(path)).get(f"config{workload_idx}_{dist}")
-        if rec and rec.get("source_hash") == kernel_source_hash():
+        if rec and rec.get("source_hash") == kernel_source_hash(rec["sources"]):
             return rec["dram_bytes_per_launch"]
     except Exception:
         pass
@@ -142,15 +143,17 @@ def stored_traffic(workload_idx, dist):
 
 # ------------------------------------------------------------------ reference arm: the CPU oracle
 def oracle_sample_rows(w):
-    """Rows per timed oracle call: about 1e8 logit elements (a few seconds of CPU work)."""
+    """Rows per timed oracle call: about 4e8 logit elements (several core-seconds of CPU work per call)."""
     per_row = w.classes * w.n
-    rows = max(1, min(w.rows, int(1.0e8 // per_row)))
+    rows = max(1, min(w.rows, int(4.0e8 // per_row)))
     if w.tokens_per_seq:
         rows = max(w.tokens_per_seq, rows // w.tokens_per_seq * w.tokens_per_seq)
     return min(rows, w.rows)
 
 
-def time_oracle(w, dist, steps, warmup):
+def time_oracle(w, dist, steps, warmup, min_seconds=0.0):
+    """Times the oracle as it stands on a bounded sample; with min_seconds the call is repeated until
+    that much wall time has been spent (at least `steps` calls)."""
     import oracle
     from paper_2010_02838_b200 import synth
     rows = oracle_sample_rows(w)
@@ -160,10 +163,12 @@ def time_oracle(w, dist, steps, warmup):
     for _ in range(warmup):
         oracle.codistill(own, peers, labels, mask, **kw)
     t0 = time.perf_counter()
-    for _ in range(steps):
+    done = 0
+    while done < steps or (time.perf_counter() - t0) < min_seconds:
         oracle.codistill(own, peers, labels, mask, **kw)
-    dt = (time.perf_counter() - t0) / max(steps, 1)
-    return rows / dt, dt, rows, oracle.max_threads()
+        done += 1
+    dt = (time.perf_counter() - t0) / max(done, 1)
+    return rows / dt, dt, rows, oracle.max_threads(), done
 
 
 def run_reference(args):
@@ -175,7 +180,7 @@ def run_reference(args):
     if args.rows:
         w = synth.scaled(w, rows=args.rows)
     steps, warmup = max(1, args.steps), max(0, args.warmup)
-    value, dt, rows, cores = time_oracle(w, args.dist, steps, warmup)
+    value, dt, rows, cores, _ = time_oracle(w, args.dist, steps, warmup)
     sample = f"first {rows} rows of the workload per step, all {w.n} models, fp64 oracle as it stands"
     line = {
         "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus, "steps": steps,
@@ -307,9 +312,10 @@ def run_ours(args):
         "clocks": clocks, "e2e": e2e, "gpu_launches": launches_per_step * args.steps,
     }
     if not args.no_cpu_baseline:
-        v, dt, rows, cores = time_oracle(w0, args.dist, 2, 1)
+        v, dt, rows, cores, calls = time_oracle(w0, args.dist, 2, 1, min_seconds=12.0)
         line["cpu_baseline"] = {"value": v, "unit": UNIT, "cores": cores, "kind": "oracle",
-                                "sample": f"first {rows} rows of the workload, all {w.n} models, {dt:.2f} s per call"}
+                                "sample": f"first {rows} rows of the workload, all {w.n} models, {calls} calls of {dt:.2f} s "
+                                          f"({calls * dt * cores:.0f} core-seconds)"}
     print(json.dumps(line), flush=True)
     if world > 1:
         dist_pkg.destroy_process_group()

@@ -17,6 +17,10 @@
 // of an unaligned row are done element by element by two designated threads.
 #include <type_traits>
 
+#ifndef STREAM_HINTS
+#define STREAM_HINTS 5   // bit 0: own-row loads of pass A ask L2 to keep the lines; bit 1: peer loads, bit 2: gradient stores marked evict-first
+#endif
+
 #include "common.cuh"
 #include "seg_math.cuh"
 
@@ -39,6 +43,26 @@ struct StreamShared {
   double fin[32];
   int last_flag;
 };
+
+// 16-byte global load / store with an L2 eviction policy (see make_policy_*).
+__device__ __forceinline__ uint4 ldg_policy(const uint4* p, uint64_t pol) {
+  uint4 r;
+  asm volatile("ld.global.L2::cache_hint.v4.u32 {%0,%1,%2,%3}, [%4], %5;" : "=r"(r.x), "=r"(r.y), "=r"(r.z), "=r"(r.w) : "l"(p), "l"(pol));
+  return r;
+}
+__device__ __forceinline__ void stg_policy(uint4* p, const uint4& v, uint64_t pol) {
+  asm volatile("st.global.L2::cache_hint.v4.u32 [%0], {%1,%2,%3,%4}, %5;" ::"l"(p), "r"(v.x), "r"(v.y), "r"(v.z), "r"(v.w), "l"(pol) : "memory");
+}
+__device__ __forceinline__ uint64_t make_policy_keep() {
+  uint64_t pol;
+  asm volatile("createpolicy.fractional.L2::evict_last.b64 %0, 1.0;" : "=l"(pol));
+  return pol;
+}
+__device__ __forceinline__ uint64_t make_policy_stream() {
+  uint64_t pol;
+  asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(pol));
+  return pol;
+}
 
 // First column of segment `s` of the row image whose value equals m, or INT_MAX; reads single elements.
 template <typename T>
@@ -68,6 +92,9 @@ __global__ void __launch_bounds__(stream_threads(P), stream_ctas_per_sm(P)) rows
   const bool stream_peers = (P >= 1) && (with_term || a.want_flags);
 
   wait_for_prior_grid();  // from here on the workspace header and the valid-row counts are read
+#if STREAM_HINTS
+  const uint64_t pol_keep = make_policy_keep(), pol_stream = make_policy_stream();
+#endif
   float w = 1.f;
   if (a.reduction == CODISTILL_REDUCE_MEAN_VALID) {
     const int64_t nv = total_valid(a);
@@ -130,7 +157,11 @@ __global__ void __launch_bounds__(stream_threads(P), stream_ctas_per_sm(P)) rows
       constexpr int B = decltype(nb)::value;
       uint4 rw[B];
 #pragma unroll
+#if STREAM_HINTS & 1
+      for (int u = 0; u < B; ++u) rw[u] = ldg_policy(z_img + s0 + (i0 + u) * NT, pol_keep);
+#else
       for (int u = 0; u < B; ++u) rw[u] = z_img[s0 + (i0 + u) * NT];
+#endif
       const float old_best = best;
 #pragma unroll
       for (int u = 0; u < B; ++u) {
@@ -259,7 +290,11 @@ __global__ void __launch_bounds__(stream_threads(P), stream_ctas_per_sm(P)) rows
         for (int jj = 0; jj < PG; ++jj) {
           if (j0 + jj < P) {
 #pragma unroll
+#if STREAM_HINTS & 2
+            for (int u = 0; u < B; ++u) pr[jj][u] = ldg_policy(p_img[j0 + jj] + s0 + (i0 + u) * NT, pol_stream);
+#else
             for (int u = 0; u < B; ++u) pr[jj][u] = p_img[j0 + jj][s0 + (i0 + u) * NT];
+#endif
           }
         }
 #pragma unroll
@@ -320,7 +355,11 @@ __global__ void __launch_bounds__(stream_threads(P), stream_ctas_per_sm(P)) rows
             if (2 * i + 1 == pos_y) g2[i].y -= cy;
           }
         }
+#if STREAM_HINTS & 4
+        if (g_img) stg_policy(g_img + s, SegOps<T>::pack2(g2), pol_stream);
+#else
         if (g_img) g_img[s] = SegOps<T>::pack2(g2);
+#endif
       }
     };
     {
