@@ -210,8 +210,13 @@ const char* codistill_status_string(int status);
 int codistill_version(void);
 
 /*
- * Name of the kernel regime the dispatcher picks for a problem ("warp", "block" or "tma"), so that
- * tests and benchmarks can state which kernel they exercised.  Static storage; NULL on bad arguments.
+ * Name of the kernel regime the dispatcher picks for a problem, so that tests and benchmarks can
+ * state which kernel they exercised: "warp" (rows up to 8 KiB, one warp per row), "tma" (long rows,
+ * MSE distance, own row staged in shared memory by bulk copies), "stream" (long rows, direct loads,
+ * own row read twice; MSE rows beyond 64 KiB and the KL distance) or "block" (everything else).  The
+ * answer assumes 16-byte aligned tensor bases (the long-row kernels need them).  The environment
+ * variable CODISTILL_REGIME = tma | stream | block overrides the choice where the named kernel can
+ * serve the call.  Static storage; NULL on bad arguments.
  */
 const char* codistill_kernel_regime(int n, int64_t rows, int64_t classes, int64_t row_stride, int dtype,
                                     int dist_kind, int peer_reduce);

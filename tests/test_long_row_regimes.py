@@ -86,3 +86,18 @@ def test_very_long_rows_take_the_stream_kernel():
     assert plan.regime == "stream"
     assert torch.all(g[:32].float() == 3.0) and torch.all(g[32 + rows * C:].float() == 3.0)
     assert torch.equal(g[32:32 + rows * C].view(rows, C), out.grad)
+
+
+@pytest.mark.parametrize("dtype", ["f32", "bf16"])
+@pytest.mark.parametrize("peer_reduce", [cb.PEERS_PAIRWISE_MEAN, cb.PEERS_MEAN_TARGET])
+@pytest.mark.parametrize("C,n,temperature", [(32768, 2, 1.0), (50257, 4, 2.0), (9001, 8, 0.7), (8192, 1, 3.0)])
+def test_kl_form_on_long_rows(dtype, peer_reduce, C, n, temperature):
+    """The softmax-KL distance on long rows is served by the direct-load kernel (one more pass for the
+    peers' softmax statistics)."""
+    rows = 13
+    own, peers, labels = rand_inputs(3 * C + n, rows, C, n, dtype)
+    mask = (np.arange(rows) % 5 != 3).astype(np.uint8)
+    labels[0], labels[1] = 0, C - 1
+    for reduction in (cb.REDUCE_SUM, cb.REDUCE_MEAN_VALID):
+        compare(own, peers, labels, mask, alpha=0.9, temperature=temperature, label_smoothing=0.05,
+                dist=cb.DIST_KL_SOFTMAX, peer_reduce=peer_reduce, reduction=reduction, expect_regime="stream")
