@@ -42,6 +42,9 @@ def parse_args():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--dist", default="mse", choices=["mse", "kl"])
     ap.add_argument("--rows", type=int, default=0, help="run a smaller batch of the same recipe (profiling aid)")
+    ap.add_argument("--all-models", action="store_true",
+                    help="one call computes the objectives of all n models (codistill_loss_fwd_bwd_all); rows/s then counts "
+                         "model-rows (n x rows per step)")
     ap.add_argument("--e2e-steps", type=int, default=3)
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
@@ -248,8 +251,14 @@ def run_ours(args):
         w0 = synth.scaled(w0, rows=args.rows)
     dist_code = cb.DIST_KL_SOFTMAX if args.dist == "kl" else cb.DIST_MSE_LOGITS
     w, models, labels, mask = make_device_inputs(w0, torch, seed_offset=rank)   # each rank: its own batch
-    plan = cb.Plan(models[0], models[1:], labels, mask, alpha=w.alpha, temperature=w.temperature,
-                   label_smoothing=w.label_smoothing, dist=dist_code)
+    if args.all_models:
+        if args.dist != "mse":
+            raise SystemExit("--all-models serves the MSE distance only")
+        plan = cb.AllPlan(models, labels, mask, alpha=w.alpha, label_smoothing=w.label_smoothing)
+        plan.regime = "all-models"
+    else:
+        plan = cb.Plan(models[0], models[1:], labels, mask, alpha=w.alpha, temperature=w.temperature,
+                       label_smoothing=w.label_smoothing, dist=dist_code)
     stream = torch.cuda.current_stream()
 
     def barrier():
@@ -277,14 +286,15 @@ def run_ours(args):
         dist_pkg.all_reduce(t, op=dist_pkg.ReduceOp.MAX)
         ms_total = float(t.item())
     ms_step = ms_total / args.steps
-    rows_per_s = world * w.rows / (ms_step * 1e-3)
+    rows_per_step = w.rows * (w.n if args.all_models else 1)
+    rows_per_s = world * rows_per_step / (ms_step * 1e-3)
     status = int(plan.out.status.item())
     if status != 0:
         raise RuntimeError(f"device status {status} after the timed region")
 
     # ---- end to end through the host-buffer entry point (pinned host memory, copies inside the timed region)
     e2e = None
-    if not args.no_e2e:
+    if not args.no_e2e and not args.all_models:
         e2e = run_e2e(args, w, models, labels, mask, cb, torch, world, barrier, dist_code)
 
     if rank != 0:
@@ -294,20 +304,28 @@ def run_ours(args):
 
     peak, peak_src = hbm_peak()
     alg_bytes = w.algorithmic_bytes(skip_masked_reads=True)
-    achieved = alg_bytes / (ms_step * 1e-3) / 1e9
     launches_per_step = 2   # prep kernel + main kernel (the main kernel's last CTA does the final reduction)
+    note = ("algorithmic bytes with masked-row reads skipped: n*R_valid*C*s + R*C*s + 9R; "
+            "duration = step time (prep + main kernel) from CUDA events on the launch stream")
+    if args.all_models:
+        es = 4 if w.dtype == "f32" else 2
+        r_valid = w.rows - w.n_padded
+        alg_bytes = w.n * (r_valid + w.rows) * w.classes * es + 9 * w.rows * w.n
+        launches_per_step = 3   # prep kernel + all-models kernel + final reduction of the n models
+        note = ("all n objectives per step; algorithmic bytes = every tensor read once and every gradient written "
+                "once: n*(R_valid + R)*C*s (the kernel reads each tensor twice: 3n passes; n single calls move n*(n+1))")
+    achieved = alg_bytes / (ms_step * 1e-3) / 1e9
     line = {
         "metric": METRIC, "value": rows_per_s, "unit": UNIT, "n_gpus": world, "steps": args.steps,
         "warmup": max(args.warmup, 3), "ms_per_step": ms_step, "higher_is_better": True, "scaling": "weak",
-        "vs_baseline": None, "dtype": "f32", "data": "synthetic", "config": workload_config(args.workload, w0, args.dist),
+        "vs_baseline": None, "dtype": "f32", "data": "synthetic", "config": dict(workload_config(args.workload, w0, args.dist), **({"all_models": True} if args.all_models else {})),
         "io_dtype": w.dtype, "kernel_regime": plan.regime,
         "hbm_gbs_algorithmic": achieved,
-        "hbm_gbs_dense_formula": w.algorithmic_bytes() / (ms_step * 1e-3) / 1e9,
+        "hbm_gbs_dense_formula": None if args.all_models else w.algorithmic_bytes() / (ms_step * 1e-3) / 1e9,
         "roofline": {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
-                     "traffic": stored_traffic(args.workload, args.dist), "peak_source": peak_src,
+                     "traffic": None if args.all_models else stored_traffic(args.workload, args.dist), "peak_source": peak_src,
                      "bytes_per_launch": alg_bytes,
-                     "note": "algorithmic bytes with masked-row reads skipped: n*R_valid*C*s + R*C*s + 9R; "
-                             "duration = step time (prep + main kernel) from CUDA events on the launch stream"},
+                     "note": note},
         "frac_of_nominal_8TBs": achieved / 8000.0,
         "clocks": clocks, "e2e": e2e, "gpu_launches": launches_per_step * args.steps,
     }

@@ -203,6 +203,52 @@ size_t codistill_workspace_bytes(int n, int64_t rows, int64_t classes, int dtype
  * Pass the row pitch as `classes` when row_stride > classes. */
 size_t codistill_host_workspace_bytes(int n, int64_t rows, int64_t classes, int dtype, int64_t chunk_rows);
 
+/*
+ * All models in one call: Algorithm 1 updates every model i = 1..n on the same minibatch ("for i = 1,
+ * ..., n in parallel"), and each update needs the objective with model i as "own" and the other n-1 as
+ * peers.  Done with n calls above, every logit tensor is read n times and n gradients are written:
+ * n (n + 1) tensor passes.  This entry point computes the n objectives together: the per-column sums
+ * over the models are shared, so that 3 n passes suffice (each tensor read twice, each gradient
+ * written once).  MSE-on-logits distance only.
+ *
+ *   logits        HOST array of n device pointers, each [rows, row_stride] in `dtype`, 16-byte aligned.
+ *   grad_logits   HOST array of n device pointers (same layout), or NULL = forward only.
+ *   row_loss      [n, rows] float device output (model-major), may be NULL.
+ *   reduced_loss  [n] float device output.
+ *   counters      [n, 3 + (n-1)] int64 device output, may be NULL: row i as for a single call with
+ *                 model i as own and the other models, in increasing index, as its peers.
+ *   n             2 .. CODISTILL_ALL_MAX_MODELS.
+ * Everything else as in codistill_params_t.  Results equal those of the n single calls within the
+ * stated tolerances; integer outputs are identical.
+ */
+#define CODISTILL_ALL_MAX_MODELS 8
+typedef struct codistill_all_params {
+  uint64_t struct_bytes;
+  const void* const* logits;
+  const int32_t* labels;
+  const uint8_t* mask;
+  int32_t n;
+  int32_t dtype;
+  int64_t rows;
+  int64_t classes;
+  int64_t row_stride;
+  float alpha;
+  float label_smoothing;
+  int32_t peer_reduce;
+  int32_t reduction;
+  float* row_loss;
+  float* reduced_loss;
+  void* const* grad_logits;
+  int64_t* counters;
+  int32_t* dev_status;
+  void* workspace;
+  uint64_t workspace_bytes;
+} codistill_all_params_t;
+int codistill_loss_fwd_bwd_all(const codistill_all_params_t* params, void* stream);
+
+/* Scratch size for codistill_loss_fwd_bwd_all (bytes; multiple of 256). */
+size_t codistill_all_workspace_bytes(int n, int64_t rows);
+
 /* Human-readable name of a CODISTILL_ERR_* code (static storage). */
 const char* codistill_status_string(int status);
 

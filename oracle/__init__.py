@@ -112,3 +112,11 @@ def codistill(own: np.ndarray, peers, labels: np.ndarray, mask: np.ndarray | Non
     if rc != 0:
         raise ValueError("codistill_oracle: invalid arguments")
     return OracleResult(row_loss, float(loss[0]), grad, counters, int(status[0]))
+
+
+def codistill_all(models, labels: np.ndarray, mask: np.ndarray | None = None, **options):
+    """Algorithm 1's inner loop "for i = 1..n": the objective of every model i with the other models,
+    in increasing index, as its peers.  Written out as n evaluations of the single-model definition;
+    returns the list of their results."""
+    models = list(models)
+    return [codistill(models[i], models[:i] + models[i + 1:], labels, mask, **options) for i in range(len(models))]

@@ -27,7 +27,7 @@ ERR_TOO_LARGE = 8
 
 EXPORTS = (
     "codistill_loss_fwd_bwd", "codistill_loss_fwd_bwd_ex", "codistill_loss_fwd_bwd_host",
-    "codistill_loss_fwd_bwd_static",
+    "codistill_loss_fwd_bwd_static", "codistill_loss_fwd_bwd_all", "codistill_all_workspace_bytes",
     "codistill_workspace_bytes", "codistill_host_workspace_bytes", "codistill_status_string",
     "codistill_version", "codistill_kernel_regime",
 )
@@ -55,6 +55,32 @@ class Params(ctypes.Structure):
         ("row_loss", ctypes.c_void_p),
         ("reduced_loss", ctypes.c_void_p),
         ("grad_logits", ctypes.c_void_p),
+        ("counters", ctypes.c_void_p),
+        ("dev_status", ctypes.c_void_p),
+        ("workspace", ctypes.c_void_p),
+        ("workspace_bytes", ctypes.c_uint64),
+    ]
+
+
+class AllParams(ctypes.Structure):
+    """Mirror of ``codistill_all_params_t``."""
+    _fields_ = [
+        ("struct_bytes", ctypes.c_uint64),
+        ("logits", ctypes.POINTER(ctypes.c_void_p)),
+        ("labels", ctypes.c_void_p),
+        ("mask", ctypes.c_void_p),
+        ("n", ctypes.c_int32),
+        ("dtype", ctypes.c_int32),
+        ("rows", ctypes.c_int64),
+        ("classes", ctypes.c_int64),
+        ("row_stride", ctypes.c_int64),
+        ("alpha", ctypes.c_float),
+        ("label_smoothing", ctypes.c_float),
+        ("peer_reduce", ctypes.c_int32),
+        ("reduction", ctypes.c_int32),
+        ("row_loss", ctypes.c_void_p),
+        ("reduced_loss", ctypes.c_void_p),
+        ("grad_logits", ctypes.POINTER(ctypes.c_void_p)),
         ("counters", ctypes.c_void_p),
         ("dev_status", ctypes.c_void_p),
         ("workspace", ctypes.c_void_p),
@@ -90,6 +116,10 @@ def load_library() -> ctypes.CDLL:
     lib.codistill_loss_fwd_bwd_ex.argtypes = [ctypes.POINTER(Params), vp]
     lib.codistill_loss_fwd_bwd_host.restype = i32
     lib.codistill_loss_fwd_bwd_host.argtypes = [ctypes.POINTER(Params), i64, vp]
+    lib.codistill_loss_fwd_bwd_all.restype = i32
+    lib.codistill_loss_fwd_bwd_all.argtypes = [ctypes.POINTER(AllParams), vp]
+    lib.codistill_all_workspace_bytes.restype = ctypes.c_size_t
+    lib.codistill_all_workspace_bytes.argtypes = [i32, i64]
     lib.codistill_workspace_bytes.restype = ctypes.c_size_t
     lib.codistill_workspace_bytes.argtypes = [i32, i64, i64, i32]
     lib.codistill_host_workspace_bytes.restype = ctypes.c_size_t
@@ -286,3 +316,59 @@ def codistill_loss_fwd_bwd_host(params: Params, chunk_rows: int = 0, stream: tor
     rc = load_library().codistill_loss_fwd_bwd_host(ctypes.byref(params), int(chunk_rows), _stream_ptr(stream))
     if rc != OK:
         raise CodistillError(rc)
+
+
+@dataclass
+class AllOutputs:
+    """Device tensors written by one all-models call (valid after the stream is synchronised)."""
+    row_loss: torch.Tensor        # [n, rows] float32
+    loss: torch.Tensor            # [n] float32
+    grads: list | None            # n tensors like the logits
+    counters: torch.Tensor        # [n, 3 + (n-1)] int64
+    status: torch.Tensor          # [1] int32
+
+
+class AllPlan:
+    """Pre-allocated outputs, workspace and parameter block for ``codistill_loss_fwd_bwd_all``: the
+    objectives of all n models (each with the others as its peers) in one call."""
+
+    def __init__(self, models, labels: torch.Tensor, mask: torch.Tensor | None = None, *, classes: int | None = None,
+                 alpha: float = 1.0, label_smoothing: float = 0.0, peer_reduce: int = PEERS_PAIRWISE_MEAN,
+                 reduction: int = REDUCE_MEAN_VALID, want_grad: bool = True):
+        self.lib = load_library()
+        models = list(models)
+        _require_cuda(labels, mask, *models)
+        rows, stride, C = _check_shapes(models[0], models[1:], labels, mask, classes)
+        n, dev, dt = len(models), models[0].device, dtype_code(models[0].dtype)
+        self.keep = (models, labels, mask)
+        grads = [torch.empty_strided(m.shape, m.stride(), dtype=m.dtype, device=dev) for m in models] if want_grad else None
+        self.out = AllOutputs(torch.empty((n, rows), dtype=torch.float32, device=dev),
+                              torch.empty(n, dtype=torch.float32, device=dev), grads,
+                              torch.empty((n, 3 + n - 1), dtype=torch.int64, device=dev),
+                              torch.empty(1, dtype=torch.int32, device=dev))
+        need = int(self.lib.codistill_all_workspace_bytes(n, rows))
+        self.workspace = torch.empty(max(need, 256), dtype=torch.uint8, device=dev)
+        self.ptrs = (ctypes.c_void_p * n)(*[m.data_ptr() for m in models])
+        self.gptrs = (ctypes.c_void_p * n)(*[g.data_ptr() for g in grads]) if want_grad else None
+        p = AllParams()
+        p.struct_bytes = ctypes.sizeof(AllParams)
+        p.logits = ctypes.cast(self.ptrs, ctypes.POINTER(ctypes.c_void_p))
+        p.labels = labels.data_ptr()
+        p.mask = mask.data_ptr() if mask is not None else None
+        p.n, p.dtype, p.rows, p.classes, p.row_stride = n, dt, rows, C, stride
+        p.alpha, p.label_smoothing = float(alpha), float(label_smoothing)
+        p.peer_reduce, p.reduction = int(peer_reduce), int(reduction)
+        p.row_loss = self.out.row_loss.data_ptr()
+        p.reduced_loss = self.out.loss.data_ptr()
+        p.grad_logits = ctypes.cast(self.gptrs, ctypes.POINTER(ctypes.c_void_p)) if want_grad else None
+        p.counters = self.out.counters.data_ptr()
+        p.dev_status = self.out.status.data_ptr()
+        p.workspace = self.workspace.data_ptr()
+        p.workspace_bytes = self.workspace.numel()
+        self.params = p
+
+    def run(self, stream: torch.cuda.Stream | None = None) -> AllOutputs:
+        rc = self.lib.codistill_loss_fwd_bwd_all(ctypes.byref(self.params), _stream_ptr(stream))
+        if rc != OK:
+            raise CodistillError(rc)
+        return self.out

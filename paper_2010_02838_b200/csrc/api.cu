@@ -190,6 +190,13 @@ static cudaError_t launch_prep(const KArgs& a, cudaStream_t stream) {
   return cudaGetLastError();
 }
 
+// the prep kernel for callers outside this file (the all-models entry point)
+cudaError_t launch_prep_rows(WsHeader* hdr, int64_t* partials, const int32_t* labels, const uint8_t* mask, int64_t rows,
+                             int64_t classes, cudaStream_t stream) {
+  prep_kernel<<<prep_grid(rows), 1024, 0, stream>>>(hdr, partials, labels, mask, rows, classes);
+  return cudaGetLastError();
+}
+
 static cudaError_t launch_main(const KArgs& a, int dtype, const DeviceInfo& di, cudaStream_t stream) {
   const Regime reg = pick_regime(a, dtype, di.smem_optin);
   if (reg == kRegimeTma) return launch_tma(a, dtype, di.num_sms, di.smem_optin, stream);
