@@ -377,3 +377,29 @@ def test_synth_is_counter_based_and_matches_recipe():
     assert synth.WORKLOADS[4].algorithmic_bytes() == 1610686464
     assert synth.WORKLOADS[4].algorithmic_bytes(True) == 1503338496
     assert synth.WORKLOADS[5].algorithmic_bytes() == 14821539840
+
+
+def test_all_models_loop_and_centred_identity():
+    """Algorithm 1's inner loop over the n models: model i's peers are the other models in increasing
+    index; and the closed form behind the all-models kernel, sum_{j != i} (z_i - z_j)^2 =
+    n z'_i^2 + sum_j z'_j^2 with z' centred on the mean over the models (brute force in numpy)."""
+    g = np.random.default_rng(12)
+    rows, C, n, alpha = 5, 9, 4, 0.7
+    models = [g.standard_normal((rows, C)).astype(np.float32) for _ in range(n)]
+    labels = g.integers(0, C, rows).astype(np.int32)
+    res = oracle.codistill_all(models, labels, None, alpha=alpha, reduction=oracle.REDUCE_SUM)
+    assert len(res) == n
+    z = np.stack([m.astype(np.float64) for m in models])           # [n, rows, C]
+    zc = z - z.mean(axis=0, keepdims=True)
+    q = (zc ** 2).sum(axis=0)
+    for i in range(n):
+        single = oracle.codistill(models[i], [models[j] for j in range(n) if j != i], labels, None, alpha=alpha,
+                                  reduction=oracle.REDUCE_SUM)
+        assert np.array_equal(res[i].row_loss, single.row_loss) and np.array_equal(res[i].grad, single.grad)
+        ce = oracle.codistill(models[i], [], labels, None, reduction=oracle.REDUCE_SUM).row_loss
+        d_closed = (n * zc[i] ** 2 + q).sum(axis=1) / ((n - 1) * C)
+        np.testing.assert_allclose((res[i].row_loss - ce) / alpha, d_closed, rtol=1e-12, atol=1e-14)
+        # counters: agreement with model j is equality of the first arg-maxes
+        am = z.argmax(axis=2)
+        others = [j for j in range(n) if j != i]
+        assert res[i].counters[3:].tolist() == [int((am[i] == am[j]).sum()) for j in others]
