@@ -145,9 +145,12 @@ def test_determinism_and_guard_bands(shape):
     assert np.abs(g - ref.grad).max() <= (1e-6 if dtype == "f32" else 2e-3)
 
 
-def test_host_buffer_entry_point():
-    """codistill_loss_fwd_bwd_host: host pointers in, host results out, several slices."""
+@pytest.mark.parametrize("regime,dist", [("tma", 0), ("stream", 0), ("stream", 1)])
+def test_host_buffer_entry_point(monkeypatch, regime, dist):
+    """codistill_loss_fwd_bwd_host: host pointers in, host results out, several slices (each slice is a
+    launch on a row range: served by either long-row kernel, and by the KL kernel)."""
     import ctypes
+    monkeypatch.setenv("CODISTILL_REGIME", regime)
     w = synth.scaled(synth.WORKLOADS[4], rows=96, classes=4096)
     own, peers, labels, mask = synth.make_inputs(w)
     n, rows, C = w.n, w.rows, w.classes
@@ -167,11 +170,12 @@ def test_host_buffer_entry_point():
     p.labels, p.mask = h_labels.data_ptr(), h_mask.data_ptr()
     p.n, p.dtype, p.rows, p.classes, p.row_stride = n, cb.BF16, rows, C, C
     p.alpha, p.temperature, p.label_smoothing = 1.0, 1.0, 0.1
+    p.dist_kind = dist
     p.row_loss, p.reduced_loss, p.grad_logits = h_row.data_ptr(), h_loss.data_ptr(), h_grad.data_ptr()
     p.counters, p.dev_status = h_cnt.data_ptr(), h_st.data_ptr()
     p.workspace, p.workspace_bytes = ws.data_ptr(), ws.numel()
     cb.codistill_loss_fwd_bwd_host(p, chunk)
-    ref = oracle.codistill(own, peers, labels, mask, alpha=1.0, label_smoothing=0.1)
+    ref = oracle.codistill(own, peers, labels, mask, alpha=1.0, label_smoothing=0.1, dist=dist)
     assert abs(h_loss.item() - ref.loss) <= 2e-3 * abs(ref.loss)
     assert h_cnt.tolist() == ref.counters.tolist() and h_st.item() == 0
     np.testing.assert_allclose(h_row.numpy(), ref.row_loss, rtol=2e-3)
