@@ -59,7 +59,9 @@ enum { CODISTILL_F32 = 0, CODISTILL_BF16 = 1 };
 /* form of the distillation distance D */
 enum {
   CODISTILL_DIST_MSE_LOGITS = 0, /* D(z, z') = 1/C * sum_c (z_c - z'_c)^2 (Appendix "Implementation Details") */
-  CODISTILL_DIST_KL_SOFTMAX = 1  /* D(z, z') = T^2 * KL(softmax(z'/T) || softmax(z/T)) (Section 2, earlier work) */
+  CODISTILL_DIST_KL_SOFTMAX = 1, /* D(z, z') = T^2 * KL(softmax(z'/T) || softmax(z/T)) (Section 2, earlier work) */
+  CODISTILL_DIST_MSE_CENTRED = 2 /* MSE between logits centred on their class means (Appendix "Implementation Details":
+                                    centring gave similar results): D(z, z') = 1/C * sum_c ((z_c - mean z) - (z'_c - mean z'))^2 */
 };
 
 /* how the n-1 peers enter D */

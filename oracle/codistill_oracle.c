@@ -13,7 +13,9 @@
  *   - Section 2: L is a standard supervised loss, cross-entropy here; earlier work used the
  *     KL divergence for D with alpha = 1.
  *   - Appendix "Implementation Details": D is the mean squared error between the logits of
- *     the two models, not centred.
+ *     the two models, not centred; the same passage says that centring the logits gave similar
+ *     results: the centred variant (each model's logits minus their mean over the classes before the
+ *     squared error, i.e. the variance over the classes of the difference) is dist_kind 2.
  *   - Section 3 / Section 5: the term may be omitted (non-communication steps), n = 1 is
  *     ordinary training.
  * Readings where the paper is silent (label smoothing target, padding mask, temperature and
@@ -35,7 +37,7 @@
 #endif
 
 enum { ORACLE_F32 = 0, ORACLE_BF16 = 1 };
-enum { ORACLE_DIST_MSE = 0, ORACLE_DIST_KL = 1 };
+enum { ORACLE_DIST_MSE = 0, ORACLE_DIST_KL = 1, ORACLE_DIST_MSE_CENTRED = 2 };
 enum { ORACLE_PEERS_PAIRWISE = 0, ORACLE_PEERS_MEAN_TARGET = 1 };
 enum { ORACLE_REDUCE_MEAN_VALID = 0, ORACLE_REDUCE_SUM = 1 };
 enum { ORACLE_STATUS_BAD_LABEL = 1 };
@@ -167,7 +169,20 @@ int codistill_oracle(const void* own, const void* const* peers, const int32_t* l
           if (!with_term) continue;
           for (int64_t c = 0; c < C; ++c) zbar[c] += zj[c] / (double)P;
           if (peer_reduce == ORACLE_PEERS_PAIRWISE) {
-            if (dist_kind == ORACLE_DIST_MSE) {
+            if (dist_kind == ORACLE_DIST_MSE_CENTRED) {
+              /* both logit vectors centred on their class means: D_j = 1/C sum_c ((z_c - mean z) - (z^(j)_c - mean z^(j)))^2 */
+              double mz = 0.0, mj_mean = 0.0;
+              for (int64_t c = 0; c < C; ++c) { mz += z[c]; mj_mean += zj[c]; }
+              mz /= (double)C; mj_mean /= (double)C;
+              double dj = 0.0;
+              for (int64_t c = 0; c < C; ++c) {
+                const double d = (z[c] - mz) - (zj[c] - mj_mean);
+                dj += d * d;
+                /* d(D_j)/dz_c = 2/C (d_c - mean_c d) and mean_c d = 0 after centring */
+                dD[c] += (2.0 / (double)C) * d / (double)P;
+              }
+              D += dj / (double)C / (double)P;
+            } else if (dist_kind == ORACLE_DIST_MSE) {
               /* D_j = 1/C sum_c (z_c - z^(j)_c)^2 */
               double dj = 0.0;
               for (int64_t c = 0; c < C; ++c) {
@@ -193,7 +208,18 @@ int codistill_oracle(const void* own, const void* const* peers, const int32_t* l
           }
         }
         if (with_term && peer_reduce == ORACLE_PEERS_MEAN_TARGET) {
-          if (dist_kind == ORACLE_DIST_MSE) {
+          if (dist_kind == ORACLE_DIST_MSE_CENTRED) {
+            double mz = 0.0, mb = 0.0;
+            for (int64_t c = 0; c < C; ++c) { mz += z[c]; mb += zbar[c]; }
+            mz /= (double)C; mb /= (double)C;
+            double d2 = 0.0;
+            for (int64_t c = 0; c < C; ++c) {
+              const double d = (z[c] - mz) - (zbar[c] - mb);
+              d2 += d * d;
+              dD[c] = (2.0 / (double)C) * d;
+            }
+            D = d2 / (double)C;
+          } else if (dist_kind == ORACLE_DIST_MSE) {
             double d2 = 0.0;
             for (int64_t c = 0; c < C; ++c) {
               const double d = z[c] - zbar[c];

@@ -17,7 +17,7 @@ LIB_PATH = os.path.join(_HERE, "libcodistill.so")
 
 OK = 0
 F32, BF16 = 0, 1
-DIST_MSE_LOGITS, DIST_KL_SOFTMAX = 0, 1
+DIST_MSE_LOGITS, DIST_KL_SOFTMAX, DIST_MSE_CENTRED = 0, 1, 2
 PEERS_PAIRWISE_MEAN, PEERS_MEAN_TARGET = 0, 1
 REDUCE_MEAN_VALID, REDUCE_SUM = 0, 1
 DEV_BAD_LABEL, DEV_TIMEOUT, DEV_ASSERT = 1, 2, 4

@@ -42,6 +42,7 @@ __device__ __forceinline__ void process_row(const KArgs& a, int64_t r, int lane,
   }
   const int y = a.labels[r];
   const bool kl = (a.dist == CODISTILL_DIST_KL_SOFTMAX);
+  const bool centred = (a.dist == CODISTILL_DIST_MSE_CENTRED);  // MSE between logits centred on their class means
   const bool with_term = (P >= 1 && a.alpha != 0.f);
   const float inv_T = 1.f / a.temperature;
 
@@ -85,7 +86,8 @@ __device__ __forceinline__ void process_row(const KArgs& a, int64_t r, int lane,
   // ---- peers: arg-max agreement and (KL, pairwise) softmax statistics
   uint32_t flags = (a_own == y) ? 1u : 0u;
   const bool peer_stats = with_term && kl && a.peer_reduce == CODISTILL_PEERS_PAIRWISE_MEAN;
-  if (P >= 1 && (a.want_flags || peer_stats)) {
+  const bool peer_means = with_term && centred;
+  if (P >= 1 && (a.want_flags || peer_stats || peer_means)) {
     for (int j = 0; j < P; ++j) {
       const T* __restrict__ p_row = reinterpret_cast<const T*>(a.peers[j]) + lr * a.row_stride;
       float pb = -INFINITY;
@@ -101,6 +103,18 @@ __device__ __forceinline__ void process_row(const KArgs& a, int64_t r, int lane,
       }
       Group<G>::argmax(pb, pi, scratch);
       if (pi == a_own) flags |= (2u << j);
+      if (peer_means) {  // difference of the class means: (mean z) - (mean z^(j)), the shift the centring removes
+        float sv[1] = {0.f};
+        for (int64_t k = lane; k < n_packets; k += G) {
+          float v[V];
+          load_packet<T, V>(p_row, k * V, v);
+#pragma unroll
+          for (int i = 0; i < V; ++i)
+            if (k * V + i < C) sv[0] += v[i];
+        }
+        Group<G>::sum(sv, scratch);
+        if (lane == 0) ps->max_v[j] = (sum_z - sv[0]) / (float)C;
+      }
       if (peer_stats) {
         float sj[1] = {0.f};
         for (int64_t k = lane; k < n_packets; k += G) {
@@ -114,7 +128,7 @@ __device__ __forceinline__ void process_row(const KArgs& a, int64_t r, int lane,
         if (lane == 0) { ps->max_v[j] = pb; ps->log_sum[j] = logf(sj[0]); }
       }
     }
-    if (peer_stats) {
+    if (peer_stats || peer_means) {
       if constexpr (G > 32) __syncthreads(); else __syncwarp();
     }
   }
@@ -179,9 +193,10 @@ __device__ __forceinline__ void process_row(const KArgs& a, int64_t r, int lane,
           for (int j = 0; j < P; ++j) {
             float u[V];
             load_packet<T, V>(reinterpret_cast<const T*>(a.peers[j]) + lr * a.row_stride, c0, u);
+            const float shift = centred ? ps->max_v[j] : 0.f;
 #pragma unroll
             for (int i = 0; i < V; ++i) {
-              const float d = v[i] - u[i];
+              const float d = (v[i] - u[i]) - shift;
               sd[i] += d;
               sq[i] = fmaf(d, d, sq[i]);
             }

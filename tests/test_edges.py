@@ -25,7 +25,7 @@ def rand_inputs(seed, rows, C, n, dtype, scale=1.5):
 
 @pytest.mark.parametrize("dtype", ["f32", "bf16"])
 @pytest.mark.parametrize("C", [1, 2, 7, 33, 257, 1000, 1023, 4099, 9001, 20011])
-@pytest.mark.parametrize("dist", [0, 1])
+@pytest.mark.parametrize("dist", [0, 1, 2])
 def test_ragged_class_counts(dtype, C, dist):
     rows = 37 if C < 5000 else 11
     own, peers, labels = rand_inputs(C, rows, C, 3, dtype)
@@ -67,7 +67,7 @@ def test_zero_rows_and_all_masked():
     assert out.loss.item() == 0.0 and torch.all(out.grad == 0)
 
 
-@pytest.mark.parametrize("dist", [0, 1])
+@pytest.mark.parametrize("dist", [0, 1, 2])
 def test_alpha_zero_n1_and_peer_equal_own(dist):
     own, peers, labels = rand_inputs(4, 20, 300, 3, "bf16")
     compare(own, peers, labels, None, alpha=0.0, dist=dist, reduction=1)     # term omitted, agreement still counted

@@ -15,7 +15,7 @@ import oracle
 from paper_2010_02838_b200 import synth
 
 GOLDEN = os.path.join(os.path.dirname(__file__), "golden")
-DISTS = [oracle.DIST_MSE, oracle.DIST_KL]
+DISTS = [oracle.DIST_MSE, oracle.DIST_KL, oracle.DIST_MSE_CENTRED]
 PEER_REDUCES = [oracle.PEERS_PAIRWISE, oracle.PEERS_MEAN_TARGET]
 
 
@@ -103,7 +103,7 @@ def test_gradient_row_sums(dist):
     alpha, C = 0.9, 13
     res = oracle.codistill(own, peers, labels, alpha=alpha, temperature=1.5, label_smoothing=0.2, dist=dist,
                            reduction=oracle.REDUCE_SUM)
-    if dist == oracle.DIST_KL:
+    if dist in (oracle.DIST_KL, oracle.DIST_MSE_CENTRED):   # shift-invariant distances: their gradient sums to zero
         assert res.grad.sum(1) == pytest.approx(np.zeros(4), abs=1e-13)
     else:
         zbar = sum(widen(p) for p in peers) / 3
@@ -151,7 +151,7 @@ def test_shift_behaviour_mse_and_kl():
         assert both.row_loss == pytest.approx(base.row_loss, rel=1e-12)
         assert both.grad == pytest.approx(base.grad, abs=1e-13)
         only_own = oracle.codistill(own_s, peers, labels, alpha=1.1, dist=dist, reduction=oracle.REDUCE_SUM)
-        if dist == oracle.DIST_KL:
+        if dist in (oracle.DIST_KL, oracle.DIST_MSE_CENTRED):   # centring removes a shift of the own logits
             assert only_own.row_loss == pytest.approx(base.row_loss, rel=1e-12)
         else:  # un-centred MSE: D changes by 2k mean_c(z - zbar) + k^2
             zbar = sum(to64(p) for p in peers) / len(peers)
@@ -328,6 +328,8 @@ def _torch_reference(own, peers, labels, mask, alpha, T, eps, dist, pr, red):
         for p in ps:
             if dist == oracle.DIST_MSE:
                 ds.append(F.mse_loss(z, p, reduction="none").mean(1))
+            elif dist == oracle.DIST_MSE_CENTRED:
+                ds.append(F.mse_loss(z - z.mean(1, keepdim=True), p - p.mean(1, keepdim=True), reduction="none").mean(1))
             else:
                 ds.append(T * T * F.kl_div(F.log_softmax(z / T, 1), F.log_softmax(p / T, 1), reduction="none",
                                            log_target=True).sum(1))
@@ -403,3 +405,30 @@ def test_all_models_loop_and_centred_identity():
         am = z.argmax(axis=2)
         others = [j for j in range(n) if j != i]
         assert res[i].counters[3:].tolist() == [int((am[i] == am[j]).sum()) for j in others]
+
+
+@pytest.mark.parametrize("pr", PEER_REDUCES)
+def test_centred_mse_is_the_variance_of_the_difference(pr):
+    """Appendix "Implementation Details" mentions centring the logits: with both logit vectors centred
+    on their class means, D_j = var_c(z - z^(j)) = MSE_j - (mean_c (z - z^(j)))^2, and the derivative is
+    (2/C) (d_c - mean_c d); brute force in numpy."""
+    own, peers, labels = rng_inputs(21, 5, 11, 4)
+    alpha, C, P = 0.6, 11, 3
+    kw = dict(alpha=alpha, peer_reduce=pr, reduction=oracle.REDUCE_SUM)
+    cen = oracle.codistill(own, peers, labels, dist=oracle.DIST_MSE_CENTRED, **kw)
+    ce = oracle.codistill(own, [], labels, reduction=oracle.REDUCE_SUM)
+    z = widen(own)
+    if pr == oracle.PEERS_MEAN_TARGET:
+        targets = [sum(widen(p) for p in peers) / P]
+    else:
+        targets = [widen(p) for p in peers]
+    D = np.zeros(5)
+    dD = np.zeros_like(z)
+    for t in targets:
+        d = z - t
+        D += (d ** 2).mean(1) - d.mean(1) ** 2
+        dD += (2.0 / C) * (d - d.mean(1, keepdims=True))
+    D /= len(targets)
+    dD /= len(targets)
+    np.testing.assert_allclose(cen.row_loss, ce.row_loss + alpha * D, rtol=1e-12, atol=1e-14)
+    np.testing.assert_allclose(cen.grad, ce.grad + alpha * dD, rtol=0, atol=1e-14)
