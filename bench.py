@@ -40,7 +40,7 @@ def parse_args():
     ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--workload", type=int, default=4, choices=[1, 2, 3, 4, 5])
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
-    ap.add_argument("--dist", default="mse", choices=["mse", "kl"])
+    ap.add_argument("--dist", default="mse", choices=["mse", "kl", "mse_centred"])
     ap.add_argument("--rows", type=int, default=0, help="run a smaller batch of the same recipe (profiling aid)")
     ap.add_argument("--all-models", action="store_true",
                     help="one call computes the objectives of all n models (codistill_loss_fwd_bwd_all); rows/s then counts "
@@ -162,7 +162,7 @@ def time_oracle(w, dist, steps, warmup, min_seconds=0.0):
     rows = oracle_sample_rows(w)
     own, peers, labels, mask = synth.make_inputs(w, 0, rows)
     kw = dict(alpha=w.alpha, temperature=w.temperature, label_smoothing=w.label_smoothing,
-              dist=oracle.DIST_KL if dist == "kl" else oracle.DIST_MSE)
+              dist={"mse": oracle.DIST_MSE, "kl": oracle.DIST_KL, "mse_centred": oracle.DIST_MSE_CENTRED}[dist])
     for _ in range(warmup):
         oracle.codistill(own, peers, labels, mask, **kw)
     t0 = time.perf_counter()
@@ -249,7 +249,7 @@ def run_ours(args):
     w0 = synth.WORKLOADS[args.workload]
     if args.rows:
         w0 = synth.scaled(w0, rows=args.rows)
-    dist_code = cb.DIST_KL_SOFTMAX if args.dist == "kl" else cb.DIST_MSE_LOGITS
+    dist_code = {"mse": cb.DIST_MSE_LOGITS, "kl": cb.DIST_KL_SOFTMAX, "mse_centred": cb.DIST_MSE_CENTRED}[args.dist]
     w, models, labels, mask = make_device_inputs(w0, torch, seed_offset=rank)   # each rank: its own batch
     if args.all_models:
         if args.dist != "mse":
