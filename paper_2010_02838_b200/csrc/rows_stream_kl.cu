@@ -38,6 +38,11 @@ template <> struct ExpUnits<__nv_bfloat16> {
   __device__ static float lg(float x) { return log2f(x); }
 };
 
+// exp_U of a pair whose arguments are already in U
+template <typename T>
+__device__ __forceinline__ float2 ex_pair(float2 x) { return make_float2(ExpUnits<T>::ex(x.x), ExpUnits<T>::ex(x.y)); }
+__device__ __forceinline__ float2 pair_of(float v) { return make_float2(v, v); }
+
 template <typename T, int P, bool PW>
 __global__ void __launch_bounds__(stream_threads(P), stream_ctas_per_sm(P)) rows_stream_kl_kernel(const __grid_constant__ KArgs a) {
   using EU = ExpUnits<T>;
@@ -64,6 +69,7 @@ __global__ void __launch_bounds__(stream_threads(P), stream_ctas_per_sm(P)) rows
   const float inv_C = 1.f / (float)C;
   const float temp = a.temperature, inv_T = 1.f / a.temperature;
   const float k1 = EU::kU, kT = EU::kU * inv_T;  // logit -> exponent argument at temperature 1 / T
+  const bool t_one = (a.temperature == 1.f);      // softmax(z / T) is softmax(z): its exponentials are shared
 
   if (tid == 0) sh.next_row[0] = a.row_begin + (long long)atomicAdd(&a.hdr->next_row, 1u);
   __syncthreads();
@@ -134,19 +140,51 @@ __global__ void __launch_bounds__(stream_threads(P), stream_ctas_per_sm(P)) rows
         }
       }
     };
-    for (int i0 = 0; i0 < cnt; i0 += kBatchA) {
-      uint4 rw[kBatchA];
+    {
+      // segments wholly inside the row: packed pairs, several loads in flight; sums relative to the running maximum
+      float2 s1p = make_float2(0.f, 0.f), sTp = make_float2(0.f, 0.f), zsp = make_float2(0.f, 0.f);
+      const float2 k1_2 = pair_of(k1), kT_2 = pair_of(kT);
+      for (int i0 = 0; i0 < cnt; i0 += kBatchA) {
+        uint4 rw[kBatchA];
 #pragma unroll
-      for (int u = 0; u < kBatchA; ++u)
-        if (i0 + u < cnt) rw[u] = ldg_policy(z_img + s0 + (i0 + u) * NT, pol_keep);
+        for (int u = 0; u < kBatchA; ++u)
+          if (i0 + u < cnt) rw[u] = ldg_policy(z_img + s0 + (i0 + u) * NT, pol_keep);
+        const float old = best;
 #pragma unroll
-      for (int u = 0; u < kBatchA; ++u) {
-        if (i0 + u < cnt) {
-          float zv[V];
-          SegOps<T>::unpack(rw[u], zv);
-          own_values(zv, s0 + (i0 + u) * NT);
+        for (int u = 0; u < kBatchA; ++u) {
+          if (i0 + u < cnt) {
+            const float fm = SegOps<T>::to_float(SegOps<T>::fold(rw[u]));
+            if (fm > best) { best = fm; best_seg = s0 + (i0 + u) * NT; }
+          }
+        }
+        const float sc1 = EU::ex((old - best) * k1);
+        s1p = __fmul2_rn(s1p, pair_of(sc1));
+        s_1 *= sc1;
+        const float2 nb1 = pair_of(-best * k1);
+        float2 nbT = nb1;
+        if (!t_one) {
+          const float scT = EU::ex((old - best) * kT);
+          sTp = __fmul2_rn(sTp, pair_of(scT));
+          s_T *= scT;
+          nbT = pair_of(-best * kT);
+        }
+#pragma unroll
+        for (int u = 0; u < kBatchA; ++u) {
+          if (i0 + u < cnt) {
+            float2 z2[H];
+            SegOps<T>::unpack2(rw[u], z2);
+#pragma unroll
+            for (int i = 0; i < H; ++i) {
+              s1p = __fadd2_rn(s1p, ex_pair<T>(__ffma2_rn(z2[i], k1_2, nb1)));
+              if (!t_one) sTp = __fadd2_rn(sTp, ex_pair<T>(__ffma2_rn(z2[i], kT_2, nbT)));
+              zsp = __fadd2_rn(zsp, z2[i]);
+            }
+          }
         }
       }
+      s_1 += s1p.x + s1p.y;
+      s_T += sTp.x + sTp.y;
+      z_sum += zsp.x + zsp.y;
     }
     if (edge) {
       float zv[V];
@@ -180,6 +218,7 @@ __global__ void __launch_bounds__(stream_threads(P), stream_ctas_per_sm(P)) rows
         S_T += sh.red_t[par][wv] * EU::ex((pt.x - m) * kT);
         sum_z += pt.w;
       }
+      if (t_one) S_T = S;
     }
     if (m_seg >= g.n_seg) m_seg = 0;  // NaN rows: keep the reads below inside the row
     const int a_own = first_equal_global<T>(z_row, m_seg, g.head, C, m);
@@ -204,33 +243,53 @@ __global__ void __launch_bounds__(stream_threads(P), stream_ctas_per_sm(P)) rows
           if (pv[i] != -INFINITY) acc += EU::ex((pv[i] - pb[q]) * kT);
         pa[q] = acc;
       };
-      for (int i0 = 0; i0 < cnt; ++i0) {
-        const int s = s0 + i0 * NT;
-        uint4 pr[PD];
+      {
+        // segments wholly inside the row: packed pairs; pa2[q] is relative to the running maximum pb[q]
+        float2 pa2[NS];
 #pragma unroll
-        for (int j = 0; j < P; ++j) pr[j] = ldg_policy(p_img[j] + s, pol_keep);
-        if constexpr (PW) {
+        for (int q = 0; q < NS; ++q) pa2[q] = make_float2(0.f, 0.f);
+        const float2 kT_2 = pair_of(kT), invP2 = pair_of(inv_P);
+        auto peer_pairs = [&](const float2 (&x2)[H], int q) {
+          float fm = fmaxf(x2[0].x, x2[0].y);
 #pragma unroll
-          for (int j = 0; j < P; ++j) {
-            float pv[V];
-            SegOps<T>::unpack(pr[j], pv);
-            peer_values(pv, j);
+          for (int i = 1; i < H; ++i) fm = fmaxf(fm, fmaxf(x2[i].x, x2[i].y));
+          const float old = pb[q];
+          pb[q] = fmaxf(pb[q], fm);
+          pa2[q] = __fmul2_rn(pa2[q], pair_of(EU::ex((old - pb[q]) * kT)));
+          const float2 nb = pair_of(-pb[q] * kT);
+#pragma unroll
+          for (int i = 0; i < H; ++i) pa2[q] = __fadd2_rn(pa2[q], ex_pair<T>(__ffma2_rn(x2[i], kT_2, nb)));
+        };
+        for (int i0 = 0; i0 < cnt; ++i0) {
+          const int s = s0 + i0 * NT;
+          uint4 pr[PD];
+#pragma unroll
+          for (int j = 0; j < P; ++j) pr[j] = ldg_policy(p_img[j] + s, pol_keep);
+          if constexpr (PW) {
+#pragma unroll
+            for (int j = 0; j < P; ++j) {
+              float2 v2[H];
+              SegOps<T>::unpack2(pr[j], v2);
+              peer_pairs(v2, j);
+            }
+          } else {
+            float2 zb2[H];
+#pragma unroll
+            for (int i = 0; i < H; ++i) zb2[i] = make_float2(0.f, 0.f);
+#pragma unroll
+            for (int j = 0; j < P; ++j) {
+              float2 v2[H];
+              SegOps<T>::unpack2(pr[j], v2);
+#pragma unroll
+              for (int i = 0; i < H; ++i) zb2[i] = __fadd2_rn(zb2[i], v2[i]);
+            }
+#pragma unroll
+            for (int i = 0; i < H; ++i) zb2[i] = __fmul2_rn(zb2[i], invP2);
+            peer_pairs(zb2, 0);
           }
-        } else {
-          float zb[V];
-#pragma unroll
-          for (int i = 0; i < V; ++i) zb[i] = 0.f;
-#pragma unroll
-          for (int j = 0; j < P; ++j) {
-            float pv[V];
-            SegOps<T>::unpack(pr[j], pv);
-#pragma unroll
-            for (int i = 0; i < V; ++i) zb[i] += pv[i];
-          }
-#pragma unroll
-          for (int i = 0; i < V; ++i) zb[i] *= inv_P;
-          peer_values(zb, 0);
         }
+#pragma unroll
+        for (int q = 0; q < NS; ++q) pa[q] = pa2[q].x + pa2[q].y;   // pa[q] was 0: the ragged segments come after
       }
       if (edge) {
         float zb[V];
@@ -329,38 +388,108 @@ __global__ void __launch_bounds__(stream_threads(P), stream_ctas_per_sm(P)) rows
       }
       return gv;
     };
-    for (int i0 = 0; i0 < cnt; ++i0) {
-      const int s = s0 + i0 * NT;
-      const uint4 zr = z_img[s];
-      uint4 pr[PD];
-      if (stream_peers) {
+    // segments wholly inside the row: packed pairs
+    typename SegOps<T>::macc ltp[PD], gep[PD];
 #pragma unroll
-        for (int j = 0; j < P; ++j) pr[j] = p_img[j][s];
-      }
-      float zv[V], gv[V], pvs[PD][V];
-      SegOps<T>::unpack(zr, zv);
+    for (int j = 0; j < PD; ++j) { ltp[j] = SegOps<T>::neg_inf(); gep[j] = SegOps<T>::neg_inf(); }
+    {
+      const float2 k1_2 = pair_of(k1), nc1_2 = pair_of(-c1), kT_2 = pair_of(kT), ncT_2 = pair_of(-cT);
+      const float2 cp2 = pair_of(cp), ncq2 = pair_of(-cq_smooth), cg2 = pair_of(cg), nts2 = pair_of(-t_scale);
+      const float2 invS2 = pair_of(__frcp_rn(S)), invP2 = pair_of(inv_P), neg1 = pair_of(-1.f);
+      const int seg_y = (g.head + y) / V, pos_y = (g.head + y) % V;
+      float2 dacc2 = make_float2(0.f, 0.f);
+      for (int i0 = 0; i0 < cnt; ++i0) {
+        const int s = s0 + i0 * NT;
+        const uint4 zr = z_img[s];
+        uint4 pr[PD];
+        if (stream_peers) {
 #pragma unroll
-      for (int j = 0; j < PD; ++j) {
-        if (stream_peers && j < P) SegOps<T>::unpack(pr[j], pvs[j]);
-        else {
-#pragma unroll
-          for (int i = 0; i < V; ++i) pvs[j][i] = 0.f;
+          for (int j = 0; j < P; ++j) pr[j] = p_img[j][s];
         }
-      }
-      const int64_t cbase = (int64_t)s * V - g.head;
+        float2 z2[H], g2[H], lp2[H], pT2[H];
+        SegOps<T>::unpack2(zr, z2);
 #pragma unroll
-      for (int i = 0; i < V; ++i) {
-        float pv[PD];
+        for (int i = 0; i < H; ++i) {
+          const float2 e = ex_pair<T>(__ffma2_rn(z2[i], k1_2, nc1_2));
+          lp2[i] = __ffma2_rn(z2[i], kT_2, ncT_2);
+          g2[i] = __ffma2_rn(e, cp2, ncq2);
+          pT2[i] = e;
+          if (with_term) pT2[i] = t_one ? __fmul2_rn(e, invS2) : ex_pair<T>(lp2[i]);
+        }
+        if (with_term) {
+          float2 ts2[H];
 #pragma unroll
-        for (int j = 0; j < PD; ++j) pv[j] = pvs[j][i];
-        gv[i] = column(zv[i], pv, cbase + i);
-      }
-      if (g_img) {
-        float2 g2[H];
+          for (int i = 0; i < H; ++i) ts2[i] = make_float2(0.f, 0.f);
+          if constexpr (PW) {
 #pragma unroll
-        for (int i = 0; i < H; ++i) g2[i] = make_float2(gv[2 * i], gv[2 * i + 1]);
-        g_img[s] = SegOps<T>::pack2(g2);
+            for (int j = 0; j < P; ++j) {
+              float2 v2[H];
+              SegOps<T>::unpack2(pr[j], v2);
+              const float2 ncq_j = pair_of(-cq[j]);
+#pragma unroll
+              for (int i = 0; i < H; ++i) {
+                const float2 l = __ffma2_rn(v2[i], kT_2, ncq_j);
+                const float2 t = ex_pair<T>(l);
+                ts2[i] = __fadd2_rn(ts2[i], t);
+                dacc2 = __ffma2_rn(t, __ffma2_rn(lp2[i], neg1, l), dacc2);
+              }
+            }
+          } else {
+            float2 zb2[H];
+#pragma unroll
+            for (int i = 0; i < H; ++i) zb2[i] = make_float2(0.f, 0.f);
+#pragma unroll
+            for (int j = 0; j < P; ++j) {
+              float2 v2[H];
+              SegOps<T>::unpack2(pr[j], v2);
+#pragma unroll
+              for (int i = 0; i < H; ++i) zb2[i] = __fadd2_rn(zb2[i], v2[i]);
+            }
+            const float2 ncq_0 = pair_of(-cq[0]);
+#pragma unroll
+            for (int i = 0; i < H; ++i) {
+              const float2 l = __ffma2_rn(__fmul2_rn(zb2[i], invP2), kT_2, ncq_0);
+              const float2 t = ex_pair<T>(l);
+              ts2[i] = t;
+              dacc2 = __ffma2_rn(t, __ffma2_rn(lp2[i], neg1, l), dacc2);
+            }
+          }
+#pragma unroll
+          for (int i = 0; i < H; ++i) g2[i] = __ffma2_rn(__ffma2_rn(ts2[i], nts2, pT2[i]), cg2, g2[i]);
+        }
+        if (a.want_flags) {
+#pragma unroll
+          for (int j = 0; j < P; ++j) {
+            const typename SegOps<T>::macc f = SegOps<T>::fold(pr[j]);
+            const bool before = s < seg_a;
+            ltp[j] = before ? SegOps<T>::mmax(ltp[j], f) : ltp[j];
+            gep[j] = before ? gep[j] : SegOps<T>::mmax(gep[j], f);
+            if (s == seg_a) {
+              // The segment of the own arg-max column a went to ge as a whole.  The peer's value at a and the
+              // largest value before a inside the segment settle the rest (see rows_stream.cu).
+              float vv[V];
+              SegOps<T>::unpack(pr[j], vv);
+              float pre = -INFINITY;
+#pragma unroll
+              for (int i = 0; i < V; ++i) {
+                const int c = seg_a * V - g.head + i;
+                if (c < a_own) pre = fmaxf(pre, vv[i]);
+                if (c == a_own) za[j] = vv[i];
+              }
+              lt[j] = fmaxf(lt[j], pre);
+            }
+          }
+        }
+        if (s == seg_y) {  // the label column: q_y carries the extra 1 - eps
+#pragma unroll
+          for (int i = 0; i < H; ++i) {
+            if (2 * i == pos_y) g2[i].x -= cy;
+            if (2 * i + 1 == pos_y) g2[i].y -= cy;
+          }
+        }
+        if (g_img) g_img[s] = SegOps<T>::pack2(g2);
       }
+      dacc += dacc2.x + dacc2.y;
     }
     if (edge) {
 #pragma unroll
@@ -381,8 +510,8 @@ __global__ void __launch_bounds__(stream_threads(P), stream_ctas_per_sm(P)) rows
       part[0] = warp_sum(dacc);
 #pragma unroll
       for (int j = 0; j < PD; ++j) {
-        part[1 + 3 * j] = warp_max_redux(lt[j]);
-        part[2 + 3 * j] = warp_max_redux(ge[j]);
+        part[1 + 3 * j] = warp_max_redux(fmaxf(lt[j], SegOps<T>::to_float(ltp[j])));
+        part[2 + 3 * j] = warp_max_redux(fmaxf(ge[j], SegOps<T>::to_float(gep[j])));
         part[3 + 3 * j] = warp_max_redux(za[j]);
       }
       if (lane == 0) {
