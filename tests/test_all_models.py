@@ -119,3 +119,27 @@ def test_all_models_equals_single_calls():
         diff = (single.grad.float() - out.grads[i].float()).abs()
         step = torch.maximum(single.grad.float().abs(), out.grads[i].float().abs()) * 2.0 ** -7
         assert bool(torch.all(diff <= step + 1e-6))
+
+
+def test_all_models_determinism_and_untouched_padding():
+    """Two runs are bit-identical; with a row pitch the padding columns of the gradients are never written."""
+    rows, C, stride, n = 23, 5001, 5008, 3
+    models, labels = rand_models(4, rows, stride, n, "bf16")
+    labels = labels % C
+    mask = (np.arange(rows) % 4 != 1).astype(np.uint8)
+    d = [to_device(m) for m in models]
+    plan = cb.AllPlan([m[:, :C] for m in d], to_device(labels), to_device(mask), classes=C, alpha=1.0,
+                      reduction=cb.REDUCE_SUM)
+    for g in plan.out.grads:   # fill the whole storage, padding columns included
+        g.as_strided(((rows - 1) * stride + C,), (1,)).fill_(7.0)
+    out = plan.run()
+    torch.cuda.synchronize()
+    first = ([g.clone() for g in out.grads], out.row_loss.clone(), out.loss.clone(), out.counters.clone())
+    out = plan.run()
+    torch.cuda.synchronize()
+    for g0, g1 in zip(first[0], out.grads):
+        assert torch.equal(g0, g1)
+        assert g1.stride(0) == stride
+        pad = g1.as_strided((rows - 1, stride), (stride, 1))[:, C:]     # the last row has no padding behind it
+        assert torch.all(pad.float() == 7.0)
+    assert torch.equal(first[1], out.row_loss) and torch.equal(first[2], out.loss) and torch.equal(first[3], out.counters)
