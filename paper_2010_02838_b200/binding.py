@@ -78,6 +78,8 @@ class AllParams(ctypes.Structure):
         ("label_smoothing", ctypes.c_float),
         ("peer_reduce", ctypes.c_int32),
         ("reduction", ctypes.c_int32),
+        ("dist_kind", ctypes.c_int32),
+        ("reserved", ctypes.c_int32),
         ("row_loss", ctypes.c_void_p),
         ("reduced_loss", ctypes.c_void_p),
         ("grad_logits", ctypes.POINTER(ctypes.c_void_p)),
@@ -333,8 +335,8 @@ class AllPlan:
     objectives of all n models (each with the others as its peers) in one call."""
 
     def __init__(self, models, labels: torch.Tensor, mask: torch.Tensor | None = None, *, classes: int | None = None,
-                 alpha: float = 1.0, label_smoothing: float = 0.0, peer_reduce: int = PEERS_PAIRWISE_MEAN,
-                 reduction: int = REDUCE_MEAN_VALID, want_grad: bool = True):
+                 alpha: float = 1.0, label_smoothing: float = 0.0, dist: int = DIST_MSE_LOGITS,
+                 peer_reduce: int = PEERS_PAIRWISE_MEAN, reduction: int = REDUCE_MEAN_VALID, want_grad: bool = True):
         self.lib = load_library()
         models = list(models)
         _require_cuda(labels, mask, *models)
@@ -357,7 +359,7 @@ class AllPlan:
         p.mask = mask.data_ptr() if mask is not None else None
         p.n, p.dtype, p.rows, p.classes, p.row_stride = n, dt, rows, C, stride
         p.alpha, p.label_smoothing = float(alpha), float(label_smoothing)
-        p.peer_reduce, p.reduction = int(peer_reduce), int(reduction)
+        p.peer_reduce, p.reduction, p.dist_kind = int(peer_reduce), int(reduction), int(dist)
         p.row_loss = self.out.row_loss.data_ptr()
         p.reduced_loss = self.out.loss.data_ptr()
         p.grad_logits = ctypes.cast(self.gptrs, ctypes.POINTER(ctypes.c_void_p)) if want_grad else None

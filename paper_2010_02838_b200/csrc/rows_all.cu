@@ -1,6 +1,7 @@
 // All n models in one call (Algorithm 1's loop "for i = 1..n in parallel" over one minibatch):
 // every model's objective with the other n-1 models as its peers, MSE-on-logits distance.
 //
+// (With the centred distance every model's logits first lose their mean over the classes, known after pass A.)
 // Per column c the n logits z_1..z_n of a row are centred on their mean mu_c, z'_i = z_i - mu_c.  Then
 //   z_i - zbar_(-i)            = n / (n-1) * z'_i                        (zbar_(-i): mean of the other models)
 //   sum_{j != i} (z_i - z_j)^2 = n * z'_i^2 + sum_j z'_j^2               (no cancellation: all terms >= 0)
@@ -37,6 +38,7 @@ struct AllArgs {
   int32_t* dev_status;          // nullable
   int64_t rows, classes, row_stride;
   int n, peer_reduce, reduction;
+  int centred;                  // distance between logits centred on their class means
   float alpha, eps;
 };
 
@@ -198,7 +200,7 @@ __global__ void __launch_bounds__(all_threads(N), all_ctas_per_sm(N)) rows_all_k
       if (lane == 0) sh.red[par][i][warp] = make_float4(m_w, __int_as_float(seg_w), sw, zw);
     }
     __syncthreads();
-    float mi[N], cpi[N];  // per model: maximum, w / S
+    float mi[N], cpi[N], cmi[N];  // per model: maximum, w / S, class mean removed before the distance (0: plain MSE)
     int a_own[N];
 #pragma unroll
     for (int i = 0; i < N; ++i) {
@@ -217,6 +219,7 @@ __global__ void __launch_bounds__(all_threads(N), all_ctas_per_sm(N)) rows_all_k
       a_own[i] = first_equal_global<T>(z_row[i], m_seg, g.head, C, m);
       mi[i] = m;
       cpi[i] = w * __frcp_rn(S);
+      cmi[i] = a.centred ? sum_z * inv_C : 0.f;
       if (tid == 0) {
         AllRowStat st;
         st.m = m; st.S = S; st.sum_z = sum_z; st.zy = Elem<T>::to_f32(z_row[i][y]); st.a_own = a_own[i];
@@ -230,13 +233,12 @@ __global__ void __launch_bounds__(all_threads(N), all_ctas_per_sm(N)) rows_all_k
     for (int i = 0; i < N; ++i) dist[i] = 0.f;
     // one column: values zc[] of the n models; returns the gradient elements in gc[]
     auto column = [&](const float (&zc)[N], float (&gc)[N], int64_t c) {
-      float mu = 0.f;
+      float zp[N], mu = 0.f, q = 0.f;
 #pragma unroll
-      for (int i = 0; i < N; ++i) mu += zc[i];
+      for (int i = 0; i < N; ++i) { zp[i] = zc[i] - cmi[i]; mu += zp[i]; }
       mu *= (1.f / (float)N);
-      float zp[N], q = 0.f;
 #pragma unroll
-      for (int i = 0; i < N; ++i) { zp[i] = zc[i] - mu; q = fmaf(zp[i], zp[i], q); }
+      for (int i = 0; i < N; ++i) { zp[i] -= mu; q = fmaf(zp[i], zp[i], q); }
       const float cqc = (c == (int64_t)y) ? cq + cy : cq;
 #pragma unroll
       for (int i = 0; i < N; ++i) {
@@ -412,6 +414,7 @@ extern "C" int codistill_loss_fwd_bwd_all(const codistill_all_params_t* p, void*
   if (!isfinite(p->alpha) || !(p->label_smoothing >= 0.f && p->label_smoothing < 1.f)) return CODISTILL_ERR_PARAM;
   if (p->peer_reduce != CODISTILL_PEERS_PAIRWISE_MEAN && p->peer_reduce != CODISTILL_PEERS_MEAN_TARGET) return CODISTILL_ERR_PARAM;
   if (p->reduction != CODISTILL_REDUCE_MEAN_VALID && p->reduction != CODISTILL_REDUCE_SUM) return CODISTILL_ERR_PARAM;
+  if (p->dist_kind != CODISTILL_DIST_MSE_LOGITS && p->dist_kind != CODISTILL_DIST_MSE_CENTRED) return CODISTILL_ERR_UNSUPPORTED;
   if (p->reduced_loss == nullptr || p->logits == nullptr) return CODISTILL_ERR_NULL;
   if (p->rows > 0 && p->labels == nullptr) return CODISTILL_ERR_NULL;
   uintptr_t bits = 0;
@@ -451,6 +454,7 @@ extern "C" int codistill_loss_fwd_bwd_all(const codistill_all_params_t* p, void*
   a.n = p->n;
   a.peer_reduce = p->peer_reduce;
   a.reduction = p->reduction;
+  a.centred = p->dist_kind == CODISTILL_DIST_MSE_CENTRED;
   a.alpha = p->alpha;
   a.eps = p->label_smoothing;
 

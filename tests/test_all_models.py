@@ -23,18 +23,18 @@ def rand_models(seed, rows, C, n, dtype, scale=1.5, spread=0.7):
     return models, labels
 
 
-def compare_all(models, labels, mask, *, classes=None, alpha=1.0, label_smoothing=0.0, peer_reduce=0, reduction=0):
+def compare_all(models, labels, mask, *, classes=None, alpha=1.0, label_smoothing=0.0, peer_reduce=0, reduction=0, dist=0):
     kind = "f32" if models[0].dtype == np.float32 else "bf16"
     tol = TOL[kind]
     C = models[0].shape[1] if classes is None else classes
     d_models = [to_device(m) for m in models]
     views = [m[:, :C] for m in d_models] if C != models[0].shape[1] else d_models
     plan = cb.AllPlan(views, to_device(labels), to_device(mask), classes=classes, alpha=alpha,
-                      label_smoothing=label_smoothing, peer_reduce=peer_reduce, reduction=reduction)
+                      label_smoothing=label_smoothing, peer_reduce=peer_reduce, reduction=reduction, dist=dist)
     out = plan.run()
     torch.cuda.synchronize()
     refs = oracle.codistill_all(models, labels, mask, classes=classes, alpha=alpha, label_smoothing=label_smoothing,
-                                peer_reduce=peer_reduce, reduction=reduction)
+                                peer_reduce=peer_reduce, reduction=reduction, dist=dist)
     counters = out.counters.cpu().numpy()
     losses = out.loss.cpu().numpy()
     rows_loss = out.row_loss.cpu().numpy().astype(np.float64)
@@ -64,8 +64,12 @@ def test_all_models_parity(dtype, n, C):
     models, labels = rand_models(100 * n + C, rows, C, n, dtype)
     mask = (np.arange(rows) % 7 != 3).astype(np.uint8)
     labels[0], labels[1] = 0, C - 1
-    for peer_reduce, reduction in ((cb.PEERS_PAIRWISE_MEAN, cb.REDUCE_SUM), (cb.PEERS_MEAN_TARGET, cb.REDUCE_MEAN_VALID)):
-        compare_all(models, labels, mask, alpha=0.8, label_smoothing=0.1, peer_reduce=peer_reduce, reduction=reduction)
+    for peer_reduce, reduction, dist in ((cb.PEERS_PAIRWISE_MEAN, cb.REDUCE_SUM, cb.DIST_MSE_LOGITS),
+                                         (cb.PEERS_MEAN_TARGET, cb.REDUCE_MEAN_VALID, cb.DIST_MSE_LOGITS),
+                                         (cb.PEERS_PAIRWISE_MEAN, cb.REDUCE_SUM, cb.DIST_MSE_CENTRED),
+                                         (cb.PEERS_MEAN_TARGET, cb.REDUCE_SUM, cb.DIST_MSE_CENTRED)):
+        compare_all(models, labels, mask, alpha=0.8, label_smoothing=0.1, peer_reduce=peer_reduce, reduction=reduction,
+                    dist=dist)
 
 
 @pytest.mark.parametrize("dtype", ["f32", "bf16"])
