@@ -22,7 +22,8 @@
 
 namespace codistill {
 
-template <typename T, int P, bool PW>
+// CEN: the centred distance (logits minus their class means): one more pass sums every peer row first.
+template <typename T, int P, bool PW, bool CEN>
 __global__ void __launch_bounds__(stream_threads(P), stream_ctas_per_sm(P)) rows_stream_kernel(const __grid_constant__ KArgs a) {
   constexpr int V = SegOps<T>::V;
   constexpr int H = SegOps<T>::H;
@@ -213,6 +214,56 @@ __global__ void __launch_bounds__(stream_threads(P), stream_ctas_per_sm(P)) rows
     for (int j = 0; j < PD; ++j)
       p_img[j] = P > 0 ? reinterpret_cast<const uint4*>(reinterpret_cast<const T*>(a.peers[j]) + row_off - g.head) : nullptr;
 
+    // centred distance: d_j = (z - mean z) - (v_j - mean v_j) = (z - v_j) - shift_j, shift_j = mean z - mean v_j
+    float2 nshift2[PD];
+    float shift[PD];
+#pragma unroll
+    for (int j = 0; j < PD; ++j) { shift[j] = 0.f; nshift2[j] = make_float2(0.f, 0.f); }
+    if constexpr (CEN && P > 0) {
+      if (with_term) {
+        float2 ps2[PD];
+        float pe[PD];
+#pragma unroll
+        for (int j = 0; j < PD; ++j) { ps2[j] = make_float2(0.f, 0.f); pe[j] = 0.f; }
+        for (int i0 = 0; i0 < cnt; ++i0) {
+          uint4 pr[PD];
+#pragma unroll
+          for (int j = 0; j < P; ++j) pr[j] = ldg_policy(p_img[j] + s0 + i0 * NT, pol_keep);
+#pragma unroll
+          for (int j = 0; j < P; ++j) {
+            float2 v2[H];
+            SegOps<T>::unpack2(pr[j], v2);
+#pragma unroll
+            for (int i = 0; i < H; ++i) ps2[j] = __fadd2_rn(ps2[j], v2[i]);
+          }
+        }
+        if (edge_head || edge_tail) {
+          const int s = edge_head ? 0 : g.n_seg - 1;
+#pragma unroll
+          for (int i = 0; i < V; ++i) {
+            const int64_t c = (int64_t)s * V - g.head + i;
+            if (c < 0 || c >= C) continue;
+#pragma unroll
+            for (int j = 0; j < P; ++j) pe[j] += Elem<T>::to_f32(reinterpret_cast<const T*>(a.peers[j])[row_off + c]);
+          }
+        }
+#pragma unroll
+        for (int j = 0; j < P; ++j) {
+          const float sw = warp_sum(ps2[j].x + ps2[j].y + pe[j]);
+          if (lane == 0) sh.cen[par][j][warp] = sw;
+        }
+        __syncthreads();
+#pragma unroll
+        for (int j = 0; j < P; ++j) {
+          float tot = 0.f;
+#pragma unroll
+          for (int wv = 0; wv < kStreamWarps; ++wv) tot += sh.cen[par][j][wv];
+          shift[j] = (sum_z - tot) * inv_C;
+          nshift2[j] = make_float2(-shift[j], -shift[j]);
+        }
+      }
+    }
+
     auto grad_batch = [&](auto nb, int i0) {
       constexpr int B = decltype(nb)::value;
       uint4 zr[B];
@@ -253,7 +304,7 @@ __global__ void __launch_bounds__(stream_threads(P), stream_ctas_per_sm(P)) rows
             SegOps<T>::unpack2(pr[jj][u], v2);
 #pragma unroll
             for (int i = 0; i < H; ++i) {
-              const float2 d = __ffma2_rn(v2[i], neg1, z2[u][i]);
+              const float2 d = CEN ? __ffma2_rn(v2[i], neg1, __fadd2_rn(z2[u][i], nshift2[j])) : __ffma2_rn(v2[i], neg1, z2[u][i]);
               if (P == 1 || j == 0) sd2[u][i] = d; else sd2[u][i] = __fadd2_rn(sd2[u][i], d);
               if constexpr (PW) { if (i & 1) dist2b = __ffma2_rn(d, d, dist2b); else dist2 = __ffma2_rn(d, d, dist2); }
             }
@@ -326,7 +377,7 @@ __global__ void __launch_bounds__(stream_threads(P), stream_ctas_per_sm(P)) rows
 #pragma unroll
           for (int j = 0; j < P; ++j) {
             const float pv = Elem<T>::to_f32(reinterpret_cast<const T*>(a.peers[j])[row_off + c]);
-            const float d = z - pv;
+            const float d = (z - pv) - shift[j];
             sd += d;
             if constexpr (PW) dist_edge = fmaf(d, d, dist_edge);
             if (a.want_flags) {
@@ -405,7 +456,7 @@ cudaError_t launch_stream_kl(const KArgs& a, int dtype, int num_sms, cudaStream_
 
 bool stream_supported(const KArgs& a, int dtype) {
   const int64_t es = dtype == CODISTILL_F32 ? 4 : 2;
-  if (a.dist != CODISTILL_DIST_MSE_LOGITS && a.dist != CODISTILL_DIST_KL_SOFTMAX) return false;
+  if (a.dist != CODISTILL_DIST_MSE_LOGITS && a.dist != CODISTILL_DIST_KL_SOFTMAX && a.dist != CODISTILL_DIST_MSE_CENTRED) return false;
   if (!(a.n_peers == 0 || a.n_peers == 1 || a.n_peers == 2 || a.n_peers == 3 || a.n_peers == 7)) return false;
   if (a.classes * es < 8192 || a.classes > (int64_t)1 << 24) return false;
   uintptr_t bits = reinterpret_cast<uintptr_t>(a.own) | reinterpret_cast<uintptr_t>(a.grad);
@@ -415,7 +466,11 @@ bool stream_supported(const KArgs& a, int dtype) {
 
 template <typename T, int P, bool PW>
 static cudaError_t stream_launch_one(const KArgs& a, int grid, cudaStream_t stream) {
-  const cudaError_t e = launch_overlapped(rows_stream_kernel<T, P, PW>, dim3(grid), dim3(stream_threads(P)), 0, stream, a);
+  cudaError_t e;
+  if (a.dist == CODISTILL_DIST_MSE_CENTRED)
+    e = launch_overlapped(rows_stream_kernel<T, P, PW, true>, dim3(grid), dim3(stream_threads(P)), 0, stream, a);
+  else
+    e = launch_overlapped(rows_stream_kernel<T, P, PW, false>, dim3(grid), dim3(stream_threads(P)), 0, stream, a);
   return e != cudaSuccess ? e : cudaGetLastError();
 }
 

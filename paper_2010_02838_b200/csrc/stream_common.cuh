@@ -23,6 +23,7 @@ __host__ __device__ constexpr int stream_ctas_per_sm(int peers) { return peers >
 struct StreamShared {
   float4 red[2][kStreamMaxWarps];                              // pass-A partials, alternating between rows
   float endred[2][kStreamMaxWarps * (1 + 3 * kStreamMaxPeers)];  // pass-B partials, alternating between rows
+  float cen[2][kStreamMaxPeers][kStreamMaxWarps];               // centred distance: per-peer class sums, alternating between rows
   long long next_row[2];
   double fin[32];
   int last_flag;

@@ -101,3 +101,19 @@ def test_kl_form_on_long_rows(dtype, peer_reduce, C, n, temperature):
     for reduction in (cb.REDUCE_SUM, cb.REDUCE_MEAN_VALID):
         compare(own, peers, labels, mask, alpha=0.9, temperature=temperature, label_smoothing=0.05,
                 dist=cb.DIST_KL_SOFTMAX, peer_reduce=peer_reduce, reduction=reduction, expect_regime="stream")
+
+
+@pytest.mark.parametrize("dtype", ["f32", "bf16"])
+@pytest.mark.parametrize("peer_reduce", [cb.PEERS_PAIRWISE_MEAN, cb.PEERS_MEAN_TARGET])
+@pytest.mark.parametrize("C,n", [(32768, 2), (50257, 4), (9001, 8), (8192, 1)])
+def test_centred_mse_on_long_rows(dtype, peer_reduce, C, n):
+    """The centred MSE distance on long rows is served by the direct-load kernel (one more pass for the
+    peers' class sums)."""
+    rows = 13
+    own, peers, labels = rand_inputs(5 * C + n, rows, C, n, dtype)
+    peers = [p if p.dtype == np.uint16 else (p + np.float32(0.5 * (j + 1))) for j, p in enumerate(peers)]  # shifted peers
+    mask = (np.arange(rows) % 5 != 3).astype(np.uint8)
+    labels[0], labels[1] = 0, C - 1
+    for reduction in (cb.REDUCE_SUM, cb.REDUCE_MEAN_VALID):
+        compare(own, peers, labels, mask, alpha=0.9, label_smoothing=0.05, dist=cb.DIST_MSE_CENTRED,
+                peer_reduce=peer_reduce, reduction=reduction, expect_regime="stream")
