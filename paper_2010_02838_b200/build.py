@@ -4,14 +4,16 @@ from __future__ import annotations
 import os
 import subprocess
 import sys
+from concurrent.futures import ThreadPoolExecutor
 
 _HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(_HERE, "csrc")
+OBJ_DIR = os.path.join(_HERE, "_build")
 LIB = os.path.join(_HERE, "libcodistill.so")
 SOURCES = ["api.cu", "rows_generic.cu", "rows_tma.cu", "rows_stream.cu", "rows_stream_kl.cu", "rows_all.cu"]
 HEADERS = ["common.cuh", "seg_math.cuh", "stream_common.cuh", os.path.join("..", "..", "include", "codistill.h")]
 NVCC_FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
-              "--shared", "-Xcompiler", "-fPIC", "-Xptxas", "-v"]
+              "-Xcompiler", "-fPIC", "-Xptxas", "-v"]
 
 
 def _stale() -> bool:
@@ -22,18 +24,33 @@ def _stale() -> bool:
     return any(os.path.getmtime(d) > t for d in deps)
 
 
+def _compile(nvcc: str, src: str):
+    obj = os.path.join(OBJ_DIR, os.path.splitext(src)[0] + ".o")
+    res = subprocess.run([nvcc, *NVCC_FLAGS, "-c", "-o", obj, os.path.join(CSRC, src)], capture_output=True, text=True)
+    return obj, res
+
+
 def build(force: bool = False, verbose: bool = False) -> str:
-    """Compile every CUDA source into one shared library (cross-compiles without a GPU)."""
+    """Compile every CUDA source (in parallel, one object per file) and link them into one shared
+    library (cross-compiles without a GPU)."""
     if force or _stale():
         nvcc = os.environ.get("NVCC", "/usr/local/cuda/bin/nvcc")
-        cmd = [nvcc, *NVCC_FLAGS, "-o", LIB, *[os.path.join(CSRC, s) for s in SOURCES]]
-        res = subprocess.run(cmd, capture_output=True, text=True)
-        if verbose or res.returncode != 0:
-            sys.stderr.write(res.stdout + res.stderr)
-        if res.returncode != 0:
+        os.makedirs(OBJ_DIR, exist_ok=True)
+        with ThreadPoolExecutor(max_workers=min(len(SOURCES), os.cpu_count() or 1)) as pool:
+            results = list(pool.map(lambda s: _compile(nvcc, s), SOURCES))
+        log = "".join(r.stdout + r.stderr for _, r in results)
+        failed = [r for _, r in results if r.returncode != 0]
+        if verbose or failed:
+            sys.stderr.write(log)
+        if failed:
             raise RuntimeError("nvcc failed building libcodistill.so")
+        link = subprocess.run([nvcc, "-gencode", "arch=compute_100a,code=sm_100a", "--shared", "-o", LIB,
+                               *[o for o, _ in results]], capture_output=True, text=True)
+        if link.returncode != 0:
+            sys.stderr.write(link.stdout + link.stderr)
+            raise RuntimeError("nvcc failed linking libcodistill.so")
         with open(os.path.join(_HERE, "build_ptxas.log"), "w") as f:
-            f.write(res.stdout + res.stderr)
+            f.write(log + link.stdout + link.stderr)
     return LIB
 
 
