@@ -252,9 +252,8 @@ def run_ours(args):
     dist_code = {"mse": cb.DIST_MSE_LOGITS, "kl": cb.DIST_KL_SOFTMAX, "mse_centred": cb.DIST_MSE_CENTRED}[args.dist]
     w, models, labels, mask = make_device_inputs(w0, torch, seed_offset=rank)   # each rank: its own batch
     if args.all_models:
-        if args.dist != "mse":
-            raise SystemExit("--all-models serves the MSE distance only")
-        plan = cb.AllPlan(models, labels, mask, alpha=w.alpha, label_smoothing=w.label_smoothing)
+        plan = cb.AllPlan(models, labels, mask, alpha=w.alpha, temperature=w.temperature,
+                          label_smoothing=w.label_smoothing, dist=dist_code)
         plan.regime = "all-models"
     else:
         plan = cb.Plan(models[0], models[1:], labels, mask, alpha=w.alpha, temperature=w.temperature,

@@ -211,8 +211,11 @@ size_t codistill_host_workspace_bytes(int n, int64_t rows, int64_t classes, int 
  * peers.  Done with n calls above, every logit tensor is read n times and n gradients are written:
  * n (n + 1) tensor passes.  This entry point computes the n objectives together: the per-column sums
  * over the models are shared, so that 3 n passes suffice (each tensor read twice, each gradient
- * written once).  MSE-on-logits distance, plain or centred (dist_kind = CODISTILL_DIST_MSE_LOGITS or
- * CODISTILL_DIST_MSE_CENTRED).
+ * written once).  Distances: MSE on logits, plain or centred (dist_kind = CODISTILL_DIST_MSE_LOGITS or
+ * CODISTILL_DIST_MSE_CENTRED), and the KL form (CODISTILL_DIST_KL_SOFTMAX, `temperature` > 0) reduced
+ * pairwise over the peers (peer_reduce = CODISTILL_PEERS_PAIRWISE_MEAN; with n = 2 the mean target is
+ * the same thing and is accepted; otherwise CODISTILL_ERR_UNSUPPORTED): the per-column sums
+ * sum_j t_j and sum_j t_j log t_j of the tempered softmaxes serve all n models.
  *
  *   logits        HOST array of n device pointers, each [rows, row_stride] in `dtype`, 16-byte aligned.
  *   grad_logits   HOST array of n device pointers (same layout), or NULL = forward only.
@@ -240,7 +243,7 @@ typedef struct codistill_all_params {
   int32_t peer_reduce;
   int32_t reduction;
   int32_t dist_kind;
-  int32_t reserved;   /* set to 0 */
+  float temperature;  /* T of the KL form; ignored by the MSE forms */
   float* row_loss;
   float* reduced_loss;
   void* const* grad_logits;

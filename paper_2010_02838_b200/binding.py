@@ -79,7 +79,7 @@ class AllParams(ctypes.Structure):
         ("peer_reduce", ctypes.c_int32),
         ("reduction", ctypes.c_int32),
         ("dist_kind", ctypes.c_int32),
-        ("reserved", ctypes.c_int32),
+        ("temperature", ctypes.c_float),
         ("row_loss", ctypes.c_void_p),
         ("reduced_loss", ctypes.c_void_p),
         ("grad_logits", ctypes.POINTER(ctypes.c_void_p)),
@@ -335,8 +335,9 @@ class AllPlan:
     objectives of all n models (each with the others as its peers) in one call."""
 
     def __init__(self, models, labels: torch.Tensor, mask: torch.Tensor | None = None, *, classes: int | None = None,
-                 alpha: float = 1.0, label_smoothing: float = 0.0, dist: int = DIST_MSE_LOGITS,
-                 peer_reduce: int = PEERS_PAIRWISE_MEAN, reduction: int = REDUCE_MEAN_VALID, want_grad: bool = True):
+                 alpha: float = 1.0, temperature: float = 1.0, label_smoothing: float = 0.0,
+                 dist: int = DIST_MSE_LOGITS, peer_reduce: int = PEERS_PAIRWISE_MEAN,
+                 reduction: int = REDUCE_MEAN_VALID, want_grad: bool = True):
         self.lib = load_library()
         models = list(models)
         _require_cuda(labels, mask, *models)
@@ -358,7 +359,7 @@ class AllPlan:
         p.labels = labels.data_ptr()
         p.mask = mask.data_ptr() if mask is not None else None
         p.n, p.dtype, p.rows, p.classes, p.row_stride = n, dt, rows, C, stride
-        p.alpha, p.label_smoothing = float(alpha), float(label_smoothing)
+        p.alpha, p.label_smoothing, p.temperature = float(alpha), float(label_smoothing), float(temperature)
         p.peer_reduce, p.reduction, p.dist_kind = int(peer_reduce), int(reduction), int(dist)
         p.row_loss = self.out.row_loss.data_ptr()
         p.reduced_loss = self.out.loss.data_ptr()

@@ -11,6 +11,12 @@
 //   pass A  the n rows: per model the online softmax statistics and the first arg-max;
 //   pass B  the n rows again: centring, distance terms, the n gradient rows.
 // Arg-max agreement between models i and j is a_i == a_j: all arg-maxes are known after pass A.
+//
+// KL distance (pairwise over the peers): with t_j = softmax(z_j / T), Q_c = sum_j t_jc and
+// E_c = sum_j t_jc log t_jc,
+//   sum_{j != i} KL(t_j || t_i)          = sum_c (E_c - Q_c log t_ic)
+//   d/dz_ic of T^2 sum_{j != i} KL(..)   = T (n t_ic - Q_c)
+// so again one read of the n rows per pass serves all n models; pass A adds sum_c exp((z - m) / T).
 #include <math.h>
 #include <string.h>
 
@@ -40,6 +46,7 @@ struct AllArgs {
   int n, peer_reduce, reduction;
   int centred;                  // distance between logits centred on their class means
   float alpha, eps;
+  float temperature;            // KL distance only
 };
 
 struct AllRowStat { float m, S, sum_z, zy; int a_own; };
@@ -47,6 +54,7 @@ struct AllRowStat { float m, S, sum_z, zy; int a_own; };
 struct AllShared {
   float4 red[2][kAllMax][kStreamMaxWarps];   // pass A partials per model: max, first segment, sum exp, sum z
   float dist[2][kAllMax][kStreamMaxWarps];   // pass B partials per model
+  float red_t[2][kAllMax][kStreamMaxWarps];  // KL: sum exp((z - m) / T) partials per model
   AllRowStat stat[2][kAllMax];
   long long next_row[2];
   double fin[32];
@@ -69,7 +77,13 @@ template <> struct WordOps<__nv_bfloat16> {
   }
 };
 
-template <typename T, int N, bool PW>
+// exp(x), x in natural units: full precision for fp32 logits, the hardware exp2 for bf16 logits
+template <typename T>
+__device__ __forceinline__ float exp_nat(float x) {
+  if constexpr (sizeof(T) == 4) return expf(x); else return ex2_approx(x * kLog2e);
+}
+
+template <typename T, int N, bool PW, bool KL>
 __global__ void __launch_bounds__(all_threads(N), all_ctas_per_sm(N)) rows_all_kernel(const __grid_constant__ AllArgs a) {
   constexpr int V = SegOps<T>::V;
   constexpr int G = WordOps<T>::G;
@@ -93,6 +107,9 @@ __global__ void __launch_bounds__(all_threads(N), all_ctas_per_sm(N)) rows_all_k
   const float cd = with_term ? w * a.alpha * (2.f * inv_C) * kRatio : 0.f;  // z'_i -> w alpha dD_i/dz_i
   const float cq = w * a.eps * inv_C;
   const float cy = w * (1.f - a.eps);
+  const float inv_T = KL ? 1.f / a.temperature : 1.f;
+  const bool t_one = a.temperature == 1.f;
+  const float ckl = with_term ? w * a.alpha * a.temperature / (float)(N - 1) : 0.f;  // (n t_i - Q) -> w alpha dD_i/dz_i
 
   if (tid == 0) sh.next_row[0] = (long long)atomicAdd(&a.hdr->next_row, 1u);
   __syncthreads();
@@ -144,11 +161,11 @@ __global__ void __launch_bounds__(all_threads(N), all_ctas_per_sm(N)) rows_all_k
     const int par = v & 1;
 
     // ================= pass A: per model, online softmax statistics and first arg-max segment
-    float best[N], s_acc[N], z_acc[N];
+    float best[N], s_acc[N], z_acc[N], t_acc[N];
     int best_seg[N];
 #pragma unroll
-    for (int i = 0; i < N; ++i) { best[i] = -3.0e38f; best_seg[i] = 0x7fffffff; s_acc[i] = 0.f; z_acc[i] = 0.f; }
-    auto stats_values = [&](const float (&zv)[V], int s, float& bst, int& bsg, float& sa, float& za) {
+    for (int i = 0; i < N; ++i) { best[i] = -3.0e38f; best_seg[i] = 0x7fffffff; s_acc[i] = 0.f; z_acc[i] = 0.f; t_acc[i] = 0.f; }
+    auto stats_values = [&](const float (&zv)[V], int s, float& bst, int& bsg, float& sa, float& za, float& ta) {
       float fm = zv[0];
 #pragma unroll
       for (int e = 1; e < V; ++e) fm = fmaxf(fm, zv[e]);
@@ -164,6 +181,14 @@ __global__ void __launch_bounds__(all_threads(N), all_ctas_per_sm(N)) rows_all_k
         }
       }
       sa = acc;
+      if constexpr (KL) {
+        if (!t_one) {
+          float acc_t = ta * exp_nat<T>((old - bst) * inv_T);
+#pragma unroll
+          for (int e = 0; e < V; ++e) acc_t += exp_nat<T>((zv[e] - bst) * inv_T);   // exp(-inf) = 0: columns outside the row
+          ta = acc_t;
+        }
+      }
     };
     for (int k = 0; k < cnt; ++k) {
       const int s = s0 + k * NT;
@@ -174,7 +199,7 @@ __global__ void __launch_bounds__(all_threads(N), all_ctas_per_sm(N)) rows_all_k
       for (int i = 0; i < N; ++i) {
         float zv[V];
         SegOps<T>::unpack(rw[i], zv);
-        stats_values(zv, s, best[i], best_seg[i], s_acc[i], z_acc[i]);
+        stats_values(zv, s, best[i], best_seg[i], s_acc[i], z_acc[i], t_acc[i]);
       }
     }
     if (edge) {
@@ -186,7 +211,7 @@ __global__ void __launch_bounds__(all_threads(N), all_ctas_per_sm(N)) rows_all_k
           const int64_t c = (int64_t)edge_seg * V - g.head + e;
           zv[e] = (c >= 0 && c < C) ? Elem<T>::to_f32(z_row[i][c]) : -INFINITY;
         }
-        stats_values(zv, edge_seg, best[i], best_seg[i], s_acc[i], z_acc[i]);
+        stats_values(zv, edge_seg, best[i], best_seg[i], s_acc[i], z_acc[i], t_acc[i]);
       }
     }
 #pragma unroll
@@ -198,9 +223,14 @@ __global__ void __launch_bounds__(all_threads(N), all_ctas_per_sm(N)) rows_all_k
       const float sw = warp_sum(s_acc[i] * rescale_exp2<T>((best[i] - m_w) * kLog2e));
       const float zw = warp_sum(z_acc[i]);
       if (lane == 0) sh.red[par][i][warp] = make_float4(m_w, __int_as_float(seg_w), sw, zw);
+      if constexpr (KL) {
+        const float tw = warp_sum(t_acc[i] * exp_nat<T>((best[i] - m_w) * inv_T));
+        if (lane == 0) sh.red_t[par][i][warp] = tw;
+      }
     }
     __syncthreads();
     float mi[N], cpi[N], cmi[N];  // per model: maximum, w / S, class mean removed before the distance (0: plain MSE)
+    float cti[KL ? N : 1], lsi[KL ? N : 1];  // KL: 1 / S_T and log S_T, S_T = sum_c exp((z_c - m) / T)
     int a_own[N];
 #pragma unroll
     for (int i = 0; i < N; ++i) {
@@ -220,6 +250,16 @@ __global__ void __launch_bounds__(all_threads(N), all_ctas_per_sm(N)) rows_all_k
       mi[i] = m;
       cpi[i] = w * __frcp_rn(S);
       cmi[i] = a.centred ? sum_z * inv_C : 0.f;
+      if constexpr (KL) {
+        float S_T = S;
+        if (!t_one) {
+          S_T = 0.f;
+#pragma unroll
+          for (int wv = 0; wv < NW; ++wv) S_T += sh.red_t[par][i][wv] * exp_nat<T>((sh.red[par][i][wv].x - m) * inv_T);
+        }
+        cti[i] = __frcp_rn(S_T);
+        lsi[i] = logf(S_T);
+      }
       if (tid == 0) {
         AllRowStat st;
         st.m = m; st.S = S; st.sum_z = sum_z; st.zy = Elem<T>::to_f32(z_row[i][y]); st.a_own = a_own[i];
@@ -233,6 +273,26 @@ __global__ void __launch_bounds__(all_threads(N), all_ctas_per_sm(N)) rows_all_k
     for (int i = 0; i < N; ++i) dist[i] = 0.f;
     // one column: values zc[] of the n models; returns the gradient elements in gc[]
     auto column = [&](const float (&zc)[N], float (&gc)[N], int64_t c) {
+      if constexpr (KL) {
+        const float cqc = (c == (int64_t)y) ? cq + cy : cq;
+        float t[N], lt[N], Q = 0.f, E = 0.f;
+#pragma unroll
+        for (int i = 0; i < N; ++i) {
+          const float x = zc[i] - mi[i];
+          const float e1 = exp_nat<T>(x);
+          t[i] = (t_one ? e1 : exp_nat<T>(x * inv_T)) * cti[i];
+          lt[i] = fmaxf(fmaf(x, inv_T, -lsi[i]), -3.0e38f);   // log t_i, kept finite so that 0 * log 0 = 0
+          Q += t[i];
+          E = fmaf(t[i], lt[i], E);
+          gc[i] = fmaf(e1, cpi[i], -cqc);
+        }
+#pragma unroll
+        for (int i = 0; i < N; ++i) {
+          gc[i] = fmaf(ckl, fmaf((float)N, t[i], -Q), gc[i]);
+          dist[i] += fmaf(-Q, lt[i], E);                       // sum_{j != i} t_j (log t_j - log t_i)
+        }
+        return;
+      }
       float zp[N], mu = 0.f, q = 0.f;
 #pragma unroll
       for (int i = 0; i < N; ++i) { zp[i] = zc[i] - cmi[i]; mu += zp[i]; }
@@ -312,7 +372,9 @@ __global__ void __launch_bounds__(all_threads(N), all_ctas_per_sm(N)) rows_all_k
       const AllRowStat st = sh.stat[par][lane];
       const float ce = (st.m + logf(st.S)) - (1.f - a.eps) * st.zy - (a.eps * inv_C) * st.sum_z;
       // pairwise: 1/((n-1) C) sum_c sum_{j != i} (z_i - z_j)^2;  mean target: 1/C sum_c (kRatio z'_i)^2
-      const float D = PW ? dsum * inv_C / (float)(N - 1) : dsum * kRatio * kRatio * inv_C;
+      // KL: T^2 / (n-1) sum_{j != i} KL(t_j || t_i)
+      const float D = KL ? a.temperature * a.temperature * dsum / (float)(N - 1)
+                         : PW ? dsum * inv_C / (float)(N - 1) : dsum * kRatio * kRatio * inv_C;
       uint32_t flags = (st.a_own == y) ? 1u : 0u;
       int bit = 1;
       for (int j = 0; j < N; ++j) {
@@ -373,10 +435,12 @@ static cudaError_t all_launch_n(const AllArgs& a, int num_sms, cudaStream_t stre
   const int64_t slots = (int64_t)num_sms * all_ctas_per_sm(N);
   const int grid = (int)(a.rows < slots ? a.rows : slots);
   cudaError_t e;
-  if (a.peer_reduce == CODISTILL_PEERS_PAIRWISE_MEAN)
-    e = launch_overlapped(rows_all_kernel<T, N, true>, dim3(grid), dim3(all_threads(N)), 0, stream, a);
+  if (a.temperature > 0.f)  // KL distance, pairwise over the peers
+    e = launch_overlapped(rows_all_kernel<T, N, true, true>, dim3(grid), dim3(all_threads(N)), 0, stream, a);
+  else if (a.peer_reduce == CODISTILL_PEERS_PAIRWISE_MEAN)
+    e = launch_overlapped(rows_all_kernel<T, N, true, false>, dim3(grid), dim3(all_threads(N)), 0, stream, a);
   else
-    e = launch_overlapped(rows_all_kernel<T, N, false>, dim3(grid), dim3(all_threads(N)), 0, stream, a);
+    e = launch_overlapped(rows_all_kernel<T, N, false, false>, dim3(grid), dim3(all_threads(N)), 0, stream, a);
   return e != cudaSuccess ? e : cudaGetLastError();
 }
 
@@ -414,7 +478,14 @@ extern "C" int codistill_loss_fwd_bwd_all(const codistill_all_params_t* p, void*
   if (!isfinite(p->alpha) || !(p->label_smoothing >= 0.f && p->label_smoothing < 1.f)) return CODISTILL_ERR_PARAM;
   if (p->peer_reduce != CODISTILL_PEERS_PAIRWISE_MEAN && p->peer_reduce != CODISTILL_PEERS_MEAN_TARGET) return CODISTILL_ERR_PARAM;
   if (p->reduction != CODISTILL_REDUCE_MEAN_VALID && p->reduction != CODISTILL_REDUCE_SUM) return CODISTILL_ERR_PARAM;
-  if (p->dist_kind != CODISTILL_DIST_MSE_LOGITS && p->dist_kind != CODISTILL_DIST_MSE_CENTRED) return CODISTILL_ERR_UNSUPPORTED;
+  if (p->dist_kind != CODISTILL_DIST_MSE_LOGITS && p->dist_kind != CODISTILL_DIST_MSE_CENTRED &&
+      p->dist_kind != CODISTILL_DIST_KL_SOFTMAX)
+    return CODISTILL_ERR_UNSUPPORTED;
+  if (p->dist_kind == CODISTILL_DIST_KL_SOFTMAX) {
+    if (!(p->temperature > 0.f) || !isfinite(p->temperature)) return CODISTILL_ERR_PARAM;
+    // the KL form is served pairwise over the peers (for n = 2 the mean target is the same thing)
+    if (p->peer_reduce != CODISTILL_PEERS_PAIRWISE_MEAN && p->n != 2) return CODISTILL_ERR_UNSUPPORTED;
+  }
   if (p->reduced_loss == nullptr || p->logits == nullptr) return CODISTILL_ERR_NULL;
   if (p->rows > 0 && p->labels == nullptr) return CODISTILL_ERR_NULL;
   uintptr_t bits = 0;
@@ -457,6 +528,7 @@ extern "C" int codistill_loss_fwd_bwd_all(const codistill_all_params_t* p, void*
   a.centred = p->dist_kind == CODISTILL_DIST_MSE_CENTRED;
   a.alpha = p->alpha;
   a.eps = p->label_smoothing;
+  a.temperature = p->dist_kind == CODISTILL_DIST_KL_SOFTMAX ? p->temperature : 0.f;  // 0: one of the MSE forms
 
   if (launch_prep_rows(a.hdr, const_cast<int64_t*>(a.partials), a.labels, a.mask, a.rows, a.classes, stream) != cudaSuccess)
     return CODISTILL_ERR_CUDA;

@@ -23,18 +23,20 @@ def rand_models(seed, rows, C, n, dtype, scale=1.5, spread=0.7):
     return models, labels
 
 
-def compare_all(models, labels, mask, *, classes=None, alpha=1.0, label_smoothing=0.0, peer_reduce=0, reduction=0, dist=0):
+def compare_all(models, labels, mask, *, classes=None, alpha=1.0, label_smoothing=0.0, peer_reduce=0, reduction=0, dist=0,
+                temperature=1.0):
     kind = "f32" if models[0].dtype == np.float32 else "bf16"
     tol = TOL[kind]
     C = models[0].shape[1] if classes is None else classes
     d_models = [to_device(m) for m in models]
     views = [m[:, :C] for m in d_models] if C != models[0].shape[1] else d_models
     plan = cb.AllPlan(views, to_device(labels), to_device(mask), classes=classes, alpha=alpha,
-                      label_smoothing=label_smoothing, peer_reduce=peer_reduce, reduction=reduction, dist=dist)
+                      label_smoothing=label_smoothing, peer_reduce=peer_reduce, reduction=reduction, dist=dist,
+                      temperature=temperature)
     out = plan.run()
     torch.cuda.synchronize()
     refs = oracle.codistill_all(models, labels, mask, classes=classes, alpha=alpha, label_smoothing=label_smoothing,
-                                peer_reduce=peer_reduce, reduction=reduction, dist=dist)
+                                peer_reduce=peer_reduce, reduction=reduction, dist=dist, temperature=temperature)
     counters = out.counters.cpu().numpy()
     losses = out.loss.cpu().numpy()
     rows_loss = out.row_loss.cpu().numpy().astype(np.float64)
@@ -70,6 +72,51 @@ def test_all_models_parity(dtype, n, C):
                                          (cb.PEERS_MEAN_TARGET, cb.REDUCE_SUM, cb.DIST_MSE_CENTRED)):
         compare_all(models, labels, mask, alpha=0.8, label_smoothing=0.1, peer_reduce=peer_reduce, reduction=reduction,
                     dist=dist)
+
+
+@pytest.mark.parametrize("dtype", ["f32", "bf16"])
+@pytest.mark.parametrize("n", [2, 3, 5, 8])
+@pytest.mark.parametrize("C", [10, 1000, 4099, 9001])
+def test_all_models_kl_parity(dtype, n, C):
+    """KL distance, pairwise over the peers, at T = 1 and T != 1."""
+    rows = 19
+    models, labels = rand_models(300 * n + C, rows, C, n, dtype)
+    mask = (np.arange(rows) % 7 != 3).astype(np.uint8)
+    labels[0], labels[1] = 0, C - 1
+    for temperature, reduction in ((1.0, cb.REDUCE_SUM), (2.0, cb.REDUCE_MEAN_VALID), (0.7, cb.REDUCE_SUM)):
+        compare_all(models, labels, mask, alpha=0.8, label_smoothing=0.1, reduction=reduction, dist=cb.DIST_KL_SOFTMAX,
+                    temperature=temperature)
+    if n == 2:   # two models: the mean target is the one peer
+        compare_all(models, labels, mask, alpha=0.8, peer_reduce=cb.PEERS_MEAN_TARGET, reduction=cb.REDUCE_SUM,
+                    dist=cb.DIST_KL_SOFTMAX, temperature=2.0)
+
+
+def test_all_models_kl_limits():
+    """Mean target with more than two models is refused; identical models give zero distance; the call
+    equals the n single-model KL calls on a workload-shaped row."""
+    rows, C, n = 8, 32768, 2
+    models, labels = rand_models(77, rows, C, n, "bf16")
+    compare_all(models, labels, None, alpha=1.0, reduction=cb.REDUCE_SUM, dist=cb.DIST_KL_SOFTMAX, temperature=2.0)
+    models3, labels3 = rand_models(78, 6, 50257, 3, "bf16")
+    compare_all(models3, labels3, None, alpha=1.0, reduction=cb.REDUCE_SUM, dist=cb.DIST_KL_SOFTMAX)
+    d = [to_device(m) for m in models3]
+    with pytest.raises(cb.CodistillError):
+        cb.AllPlan(d, to_device(labels3), None, dist=cb.DIST_KL_SOFTMAX, peer_reduce=cb.PEERS_MEAN_TARGET).run()
+    with pytest.raises(cb.CodistillError):
+        cb.AllPlan(d, to_device(labels3), None, dist=cb.DIST_KL_SOFTMAX, temperature=0.0).run()
+    same = [models3[0].copy() for _ in range(3)]
+    plan, out, refs = compare_all(same, labels3, None, alpha=2.0, reduction=cb.REDUCE_SUM, dist=cb.DIST_KL_SOFTMAX,
+                                  temperature=1.5)
+    ce_only = oracle.codistill(same[0], [], labels3, None, reduction=oracle.REDUCE_SUM)
+    assert abs(out.loss[0].item() - ce_only.loss) <= 1e-5 * abs(ce_only.loss)
+    dl = to_device(labels3)
+    allp = cb.AllPlan(d, dl, None, alpha=1.0, temperature=2.0, dist=cb.DIST_KL_SOFTMAX, reduction=cb.REDUCE_SUM).run()
+    for i in range(3):
+        single = cb.Plan(d[i], d[:i] + d[i + 1:], dl, None, alpha=1.0, temperature=2.0, dist=cb.DIST_KL_SOFTMAX,
+                         reduction=cb.REDUCE_SUM).run()
+        torch.cuda.synchronize()
+        assert single.counters.cpu().tolist() == allp.counters[i].cpu().tolist()
+        assert abs(single.loss.item() - allp.loss[i].item()) <= 1e-4 * abs(single.loss.item())
 
 
 @pytest.mark.parametrize("dtype", ["f32", "bf16"])

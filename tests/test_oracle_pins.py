@@ -407,6 +407,28 @@ def test_all_models_loop_and_centred_identity():
         assert res[i].counters[3:].tolist() == [int((am[i] == am[j]).sum()) for j in others]
 
 
+def test_all_models_kl_shared_column_sums():
+    """The closed form behind the all-models KL kernel: with t_j = softmax(z_j / T), Q = sum_j t_j and
+    E = sum_j t_j log t_j per column, sum_{j != i} KL(t_j || t_i) = sum_c (E_c - Q_c log t_ic) and the
+    derivative of T^2 times it with respect to z_i is T (n t_i - Q); brute force in numpy against the
+    oracle's pairwise loop."""
+    g = np.random.default_rng(31)
+    rows, C, n, alpha, T = 4, 13, 5, 0.9, 2.5
+    models = [(1.5 * g.standard_normal((rows, C))).astype(np.float32) for _ in range(n)]
+    labels = g.integers(0, C, rows).astype(np.int32)
+    kw = dict(alpha=alpha, temperature=T, dist=oracle.DIST_KL, reduction=oracle.REDUCE_SUM)
+    res = oracle.codistill_all(models, labels, None, **kw)
+    z = np.stack([m.astype(np.float64) for m in models]) / T
+    log_t = z - np.log(np.exp(z).sum(axis=2, keepdims=True))
+    t = np.exp(log_t)
+    Q, E = t.sum(axis=0), (t * log_t).sum(axis=0)
+    for i in range(n):
+        plain = oracle.codistill(models[i], [], labels, None, reduction=oracle.REDUCE_SUM)
+        d_closed = T * T * (E - Q * log_t[i]).sum(axis=1) / (n - 1)
+        np.testing.assert_allclose((res[i].row_loss - plain.row_loss) / alpha, d_closed, rtol=1e-11, atol=1e-13)
+        np.testing.assert_allclose((res[i].grad - plain.grad) / alpha, T * (n * t[i] - Q) / (n - 1), rtol=1e-11, atol=1e-13)
+
+
 @pytest.mark.parametrize("pr", PEER_REDUCES)
 def test_centred_mse_is_the_variance_of_the_difference(pr):
     """Appendix "Implementation Details" mentions centring the logits: with both logit vectors centred
