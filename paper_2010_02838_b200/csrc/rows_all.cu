@@ -77,8 +77,6 @@ template <> struct WordOps<__nv_bfloat16> {
   }
 };
 
-// Asks the L2 for the line that holds p (no register is tied up while it travels).
-__device__ __forceinline__ void prefetch_l2(const void* p) { asm volatile("prefetch.global.L2 [%0];" ::"l"(p)); }
 // Iterations a thread's segments are requested ahead of their loads.  The MSE forms wait on memory most of
 // the time and gain 6-15 %; the KL form is bound by arithmetic and the extra instructions cost it 3 %.
 __host__ __device__ constexpr int all_ahead(int n, bool kl) { return kl ? 0 : n >= 5 ? 1 : 2; }

@@ -30,6 +30,7 @@ __global__ void __launch_bounds__(stream_threads(P), stream_ctas_per_sm(P)) rows
   constexpr int PD = P > 0 ? P : 1;
   constexpr int ES = (int)sizeof(T);
   constexpr int NT = stream_threads(P);
+  constexpr int kAhead = stream_ahead(P);
   constexpr int kStreamWarps = NT / 32;
   __shared__ StreamShared sh;
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
@@ -101,6 +102,13 @@ __global__ void __launch_bounds__(stream_threads(P), stream_ctas_per_sm(P)) rows
     float s_edge = 0.f, z_edge = 0.f;
     auto sweep_batch = [&](auto nb, int i0) {
       constexpr int B = decltype(nb)::value;
+      if (kAhead > 0) {
+#pragma unroll
+        for (int u = 0; u < B; ++u) {
+          const int ia = i0 + kAhead * B + u;
+          if (ia < cnt) prefetch_l2(z_img + s0 + ia * NT);
+        }
+      }
       uint4 rw[B];
 #pragma unroll
 #if STREAM_HINTS & 1
@@ -266,6 +274,16 @@ __global__ void __launch_bounds__(stream_threads(P), stream_ctas_per_sm(P)) rows
 
     auto grad_batch = [&](auto nb, int i0) {
       constexpr int B = decltype(nb)::value;
+      if (kAhead > 0 && stream_peers) {  // the peers' segments of a later batch: into the L2, no register held
+#pragma unroll
+        for (int u = 0; u < B; ++u) {
+          const int ia = i0 + kAhead * B + u;
+          if (ia < cnt) {
+#pragma unroll
+            for (int j = 0; j < P; ++j) prefetch_l2(p_img[j] + s0 + ia * NT);
+          }
+        }
+      }
       uint4 zr[B];
 #pragma unroll
       for (int u = 0; u < B; ++u) zr[u] = z_img[s0 + (i0 + u) * NT];

@@ -30,6 +30,13 @@ struct StreamShared {
 };
 
 // 16-byte global load / store with an L2 eviction policy (see make_policy_*).
+// Batches of a thread's segments requested from the L2 ahead of their loads (0: none): the own row in the
+// statistics pass, the peers in the gradient pass.  One batch ahead in both is 10 % faster with one peer
+// (few independent loads in flight per thread); with seven peers it changes nothing or costs 2 %, and two
+// batches ahead were slower everywhere.
+__host__ __device__ constexpr int stream_ahead(int peers) { return peers <= 3 ? 1 : 0; }
+__device__ __forceinline__ void prefetch_l2(const void* p) { asm volatile("prefetch.global.L2 [%0];" ::"l"(p)); }
+
 __device__ __forceinline__ uint4 ldg_policy(const uint4* p, uint64_t pol) {
   uint4 r;
   asm volatile("ld.global.L2::cache_hint.v4.u32 {%0,%1,%2,%3}, [%4], %5;" : "=r"(r.x), "=r"(r.y), "=r"(r.z), "=r"(r.w) : "l"(p), "l"(pol));
