@@ -234,6 +234,10 @@ __global__ void __launch_bounds__(stream_threads(P), stream_ctas_per_sm(P)) rows
 #pragma unroll
         for (int j = 0; j < PD; ++j) { ps2[j] = make_float2(0.f, 0.f); pe[j] = 0.f; }
         for (int i0 = 0; i0 < cnt; ++i0) {
+          if (kAhead > 0 && i0 + 4 < cnt) {   // the peers' segments four iterations on: into the L2
+#pragma unroll
+            for (int j = 0; j < P; ++j) prefetch_l2(p_img[j] + s0 + (i0 + 4) * NT);
+          }
           uint4 pr[PD];
 #pragma unroll
           for (int j = 0; j < P; ++j) pr[j] = ldg_policy(p_img[j] + s0 + i0 * NT, pol_keep);
