@@ -166,11 +166,15 @@ int codistill_loss_fwd_bwd(const void* logits, const void* const* peer_logits /*
  * CODISTILL_STATIC_MAX_ROWS rows; a larger `rows` returns CODISTILL_ERR_TOO_LARGE and launches
  * nothing.  The call performs no cudaMalloc, cudaFree or other allocating routine.
  *
- * Arguments, defaults and outputs are exactly those of codistill_loss_fwd_bwd, except that
- * row_loss must not be NULL (a missing row_loss would need per-row scratch of the caller's size).
+ * Arguments, defaults and outputs are exactly those of codistill_loss_fwd_bwd (row_loss may be NULL:
+ * the per-row losses then stay inside the built-in scratch).
  *
  * Set-up: the first call on each device looks up the device address of the array (the device
- * must be current, as for every call).  Make that first call outside any stream capture.
+ * must be current, as for every call).  Make that first call outside any stream capture, and while
+ * the device still has room for this library's code and the array itself: the CUDA runtime may
+ * load both only when the library is first used on a device, so a process that fills the device
+ * memory before its first call into the library can see that call fail with CODISTILL_ERR_CUDA.
+ * Host threads may make their first calls concurrently.
  *
  * Sharing: all calls on a device use the same array, which keeps whatever the previous call left
  * in it; each call clears the words that must start at zero before using them.  Two calls that

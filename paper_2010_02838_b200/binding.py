@@ -239,8 +239,8 @@ def codistill_loss_fwd_bwd_static(logits: torch.Tensor, peer_logits, labels: tor
     """The allocation-free entry point of the C ABI.  For callers that must not touch a CUDA
     allocator at call time (all device memory already claimed by a framework, or a loop that bans
     allocator calls): the library's scratch is a fixed array in its device image, good for at most
-    ``STATIC_MAX_ROWS`` rows.  Nothing is allocated here either, so ``out`` (row_loss, loss and
-    optionally grad) must be supplied.  Calls on one device share the scratch: keep them ordered."""
+    ``STATIC_MAX_ROWS`` rows.  Nothing is allocated here either, so ``out`` (loss, and optionally row_loss
+    and grad) must be supplied.  Calls on one device share the scratch: keep them ordered."""
     lib = load_library()
     peers = list(peer_logits)
     _require_cuda(logits, labels, mask, out.row_loss, out.loss, out.grad, *peers)

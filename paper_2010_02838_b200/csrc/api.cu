@@ -4,6 +4,9 @@
 #include <stdlib.h>
 #include <string.h>
 
+#include <atomic>
+#include <mutex>
+
 #include "common.cuh"
 
 static_assert(sizeof(codistill_params_t) == 152, "ABI: size of codistill_params_t");
@@ -470,16 +473,22 @@ namespace codistill {
 constexpr size_t kStaticScratchBytes = 256 + 1024 + 2 * 4 * (size_t)CODISTILL_STATIC_MAX_ROWS;
 static __device__ __align__(256) unsigned char g_static_scratch[kStaticScratchBytes];
 
-// Device address of the scratch array on the current device, looked up once per device.
+// Device address of the scratch array on the current device, looked up once per device.  Host threads
+// may make their first calls on a device at the same time: the table is filled under a mutex and read
+// through acquire loads, so that no thread ever sees a half-published entry.
 static int static_scratch_address(void** out) {
-  static void* cache[64];
-  static bool known[64];
+  static std::atomic<void*> cache[64];
+  static std::mutex fill;
   int dev = 0;
   if (cudaGetDevice(&dev) != cudaSuccess) return CODISTILL_ERR_CUDA;
-  if (dev >= 0 && dev < 64 && known[dev]) { *out = cache[dev]; return CODISTILL_OK; }
+  const bool cached = dev >= 0 && dev < 64;
+  if (cached) {
+    if (void* known = cache[dev].load(std::memory_order_acquire)) { *out = known; return CODISTILL_OK; }
+  }
+  std::lock_guard<std::mutex> lock(fill);
   void* ptr = nullptr;
   if (cudaGetSymbolAddress(&ptr, g_static_scratch) != cudaSuccess || ptr == nullptr) return CODISTILL_ERR_CUDA;
-  if (dev >= 0 && dev < 64) { cache[dev] = ptr; known[dev] = true; }
+  if (cached) cache[dev].store(ptr, std::memory_order_release);
   *out = ptr;
   return CODISTILL_OK;
 }
@@ -513,7 +522,6 @@ extern "C" int codistill_loss_fwd_bwd_static(const void* logits, const void* con
   p.workspace = reinterpret_cast<void*>(uintptr_t(256));  // placeholder for validation; replaced below
   const int v = validate(&p, false);
   if (v != CODISTILL_OK) return v;
-  if (row_loss == nullptr) return CODISTILL_ERR_NULL;
   if (rows > (int64_t)CODISTILL_STATIC_MAX_ROWS) return CODISTILL_ERR_TOO_LARGE;
   if (ws_layout(rows).total > kStaticScratchBytes) return CODISTILL_ERR_TOO_LARGE;
   void* scratch = nullptr;

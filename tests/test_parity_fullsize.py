@@ -1,7 +1,8 @@
-"""GPU parity at the full sizes of the two large workloads, in the launch configuration bench.py
-times (MSE distance, mean over valid rows, counters on).  The oracle computes every per-row loss,
-the reduced loss and the counters for the whole batch, and the gradient for three row ranges
-(first, middle, last rows, which include padded rows)."""
+"""GPU parity at the full sizes of the two large workloads, in the launch configurations bench.py
+times (mean over valid rows, counters on): the single-model call with the MSE, softmax-KL and centred
+MSE distances, and the all-models call.  The oracle computes every per-row loss, the reduced loss and
+the counters for the whole batch, and the gradient for three row ranges (first, middle, last rows,
+which include padded rows)."""
 import numpy as np
 import pytest
 import torch
@@ -14,36 +15,97 @@ from helpers import bf16_ulp, to_device
 
 pytestmark = pytest.mark.gpu
 
+DIST = {"mse": cb.DIST_MSE_LOGITS, "kl": cb.DIST_KL_SOFTMAX, "mse_centred": cb.DIST_MSE_CENTRED}
+_cache = {}
 
-@pytest.mark.parametrize("idx", [4, 5])
-def test_full_size_workload(idx):
-    w = synth.WORKLOADS[idx]
-    free, _ = torch.cuda.mem_get_info()
-    if free < 1.3 * w.algorithmic_bytes():
-        pytest.skip("not enough free device memory for the full workload")
-    own, peers, labels, mask = synth.make_inputs(w)
-    d_own, d_peers = to_device(own), [to_device(p) for p in peers]
-    plan = cb.Plan(d_own, d_peers, to_device(labels), to_device(mask), alpha=w.alpha, temperature=w.temperature,
-                   label_smoothing=w.label_smoothing)
-    assert plan.regime == {4: "tma", 5: "stream"}[idx]      # the launch configuration the benchmark times
+
+def full_workload(idx):
+    """Host and device copies of a whole workload, generated once per test session and workload."""
+    if _cache.get("idx") != idx:
+        _cache.clear()
+        torch.cuda.empty_cache()
+        w = synth.WORKLOADS[idx]
+        free, _ = torch.cuda.mem_get_info()
+        if free < 2.6 * w.n * w.rows * w.classes * w.elem_bytes:
+            pytest.skip("not enough free device memory for the full workload")
+        own, peers, labels, mask = synth.make_inputs(w)
+        models = [own] + peers
+        _cache.update(idx=idx, w=w, models=models, labels=labels, mask=mask,
+                      d_models=[to_device(m) for m in models], d_labels=to_device(labels), d_mask=to_device(mask))
+    return _cache
+
+
+def check_gradient_rows(grad, ref_rows, mask, lo, n_valid):
+    g = grad[lo:lo + 32].double().cpu().numpy()
+    # under the mean every element is scaled by 1/n_valid: compare at that scale (values whose
+    # scaled magnitude exceeds 1 are bounded by bf16 rounding itself, as in helpers.compare)
+    err = np.abs(g - ref_rows) * n_valid
+    assert np.all(err <= np.maximum(2e-3, 0.75 * bf16_ulp(ref_rows * n_valid))), float(err.max())
+    dead = np.flatnonzero(mask[lo:lo + 32] == 0)
+    assert np.all(g[dead] == 0)
+
+
+def single_model_call(idx, dist):
+    c = full_workload(idx)
+    w, models, labels, mask = c["w"], c["models"], c["labels"], c["mask"]
+    plan = cb.Plan(c["d_models"][0], c["d_models"][1:], c["d_labels"], c["d_mask"], alpha=w.alpha,
+                   temperature=w.temperature, label_smoothing=w.label_smoothing, dist=DIST[dist])
+    if dist == "mse":
+        assert plan.regime == {4: "tma", 5: "stream"}[idx]      # the launch configuration the benchmark times
+    else:
+        assert plan.regime != "block"
     out = plan.run()
     torch.cuda.synchronize()
     assert out.status.item() == 0
-    kw = dict(alpha=w.alpha, temperature=w.temperature, label_smoothing=w.label_smoothing)
-    ref = oracle.codistill(own, peers, labels, mask, want_grad=False, **kw)
+    kw = dict(alpha=w.alpha, temperature=w.temperature, label_smoothing=w.label_smoothing, dist=DIST[dist])
+    ref = oracle.codistill(models[0], models[1:], labels, mask, want_grad=False, **kw)
     assert out.counters.cpu().tolist() == ref.counters.tolist()                  # integers: bit-exact
     assert abs(out.loss.item() - ref.loss) <= 2e-3 * abs(ref.loss)
     np.testing.assert_allclose(out.row_loss.cpu().numpy(), ref.row_loss, rtol=2e-3, atol=2e-7)
     n_valid = int(ref.counters[0])
     R = w.rows
     for lo in (0, R // 2 - 16, R - 32):
-        part = oracle.codistill(own, peers, labels, mask, grad_rows=(lo, lo + 32), **kw)
-        g = out.grad[lo:lo + 32].double().cpu().numpy()
-        # under the mean every element is scaled by 1/n_valid: compare at that scale (values whose
-        # scaled magnitude exceeds 1 are bounded by bf16 rounding itself, as in helpers.compare)
-        err = np.abs(g - part.grad) * n_valid
-        assert np.all(err <= np.maximum(2e-3, 0.75 * bf16_ulp(part.grad * n_valid)))
-        dead = np.flatnonzero(mask[lo:lo + 32] == 0)
-        assert np.all(g[dead] == 0)
-    del plan, out, d_own, d_peers
+        part = oracle.codistill(models[0], models[1:], labels, mask, grad_rows=(lo, lo + 32), **kw)
+        check_gradient_rows(out.grad, part.grad, mask, lo, n_valid)
+    del plan, out
+    torch.cuda.empty_cache()
+
+
+def all_models_call(idx, dist):
+    """Every model's objective from one call on the whole batch, against the oracle's loop over the models."""
+    c = full_workload(idx)
+    w, models, labels, mask = c["w"], c["models"], c["labels"], c["mask"]
+    plan = cb.AllPlan(c["d_models"], c["d_labels"], c["d_mask"], alpha=w.alpha, temperature=w.temperature,
+                      label_smoothing=w.label_smoothing, dist=DIST[dist])
+    out = plan.run()
+    torch.cuda.synchronize()
+    assert out.status.item() == 0
+    kw = dict(alpha=w.alpha, temperature=w.temperature, label_smoothing=w.label_smoothing, dist=DIST[dist])
+    counters, losses, row_loss = out.counters.cpu().numpy(), out.loss.cpu().numpy(), out.row_loss.cpu().numpy()
+    R = w.rows
+    for i in range(w.n):
+        peers = models[:i] + models[i + 1:]
+        ref = oracle.codistill(models[i], peers, labels, mask, want_grad=False, **kw)
+        assert counters[i].tolist() == ref.counters.tolist()
+        assert abs(losses[i] - ref.loss) <= 2e-3 * abs(ref.loss)
+        np.testing.assert_allclose(row_loss[i], ref.row_loss, rtol=2e-3, atol=2e-7)
+        n_valid = int(ref.counters[0])
+        for lo in ((0, R - 32) if i % 2 == 0 else (R // 2 - 16,)):
+            part = oracle.codistill(models[i], peers, labels, mask, grad_rows=(lo, lo + 32), **kw)
+            check_gradient_rows(out.grads[i], part.grad, mask, lo, n_valid)
+    del plan, out
+    torch.cuda.empty_cache()
+
+
+# ordered so that each workload is generated once
+@pytest.mark.parametrize("idx,call,dist", [(4, "single", "mse"), (4, "single", "kl"), (4, "single", "mse_centred"),
+                                           (4, "all", "kl"), (5, "single", "mse"), (5, "single", "kl"),
+                                           (5, "single", "mse_centred"), (5, "all", "mse"), (5, "all", "kl")])
+def test_full_size_workload(idx, call, dist):
+    (single_model_call if call == "single" else all_models_call)(idx, dist)
+
+
+def test_release_cached_workloads():
+    """Frees the device copies the tests above shared (kept last in this file)."""
+    _cache.clear()
     torch.cuda.empty_cache()
