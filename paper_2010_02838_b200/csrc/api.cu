@@ -19,6 +19,8 @@ int tma_ctas_per_sm(const KArgs& a, int dtype, int smem_optin);
 cudaError_t launch_tma(const KArgs& a, int dtype, int num_sms, int smem_optin, cudaStream_t stream);
 bool stream_supported(const KArgs& a, int dtype);
 cudaError_t launch_stream(const KArgs& a, int dtype, int num_sms, cudaStream_t stream);
+bool cluster_supported(const KArgs& a, int dtype, int smem_optin);
+cudaError_t launch_cluster_single(const KArgs& a, int dtype, int smem_optin, cudaStream_t stream);
 
 // ------------------------------------------------------------------ prep and finalize kernels
 // Zeroes the workspace header and counts valid / masked rows (one partial pair per block, summed
@@ -119,7 +121,7 @@ static int validate(const codistill_params_t* p, bool host_pointers) {
   return CODISTILL_OK;
 }
 
-enum Regime { kRegimeWarp = 0, kRegimeBlock = 1, kRegimeTma = 2, kRegimeStream = 3 };
+enum Regime { kRegimeWarp = 0, kRegimeBlock = 1, kRegimeTma = 2, kRegimeStream = 3, kRegimeCluster = 4 };
 
 // Long rows with the MSE distance have two kernels: "tma" (own row staged in shared memory by bulk
 // copies) and "stream" (direct loads, own row re-read through L2).  The staged kernel is the faster
@@ -131,11 +133,16 @@ static Regime pick_regime(const KArgs& a, int dtype, int smem_optin) {
   const int64_t row_bytes = a.classes * (dtype == CODISTILL_F32 ? 4 : 2);
   const Regime generic = row_bytes <= 8192 ? kRegimeWarp : kRegimeBlock;
   const bool can_tma = tma_supported(a, dtype, smem_optin), can_stream = stream_supported(a, dtype);
+  const bool can_cluster = cluster_supported(a, dtype, smem_optin);
   if (const char* want = getenv("CODISTILL_REGIME")) {
     if (strcmp(want, "tma") == 0 && can_tma) return kRegimeTma;
     if (strcmp(want, "stream") == 0 && can_stream) return kRegimeStream;
+    if (strcmp(want, "cluster") == 0 && can_cluster) return kRegimeCluster;
     if (strcmp(want, "block") == 0) return generic;
   }
+  // Distances whose gradient needs row statistics of the peers (softmax-KL, centred MSE) would read the
+  // peers twice from global memory: the cluster-resident kernel keeps all n rows on chip instead.
+  if (can_cluster && a.dist != CODISTILL_DIST_MSE_LOGITS) return kRegimeCluster;
   if (can_tma && (!can_stream || tma_ctas_per_sm(a, dtype, smem_optin) >= 2)) return kRegimeTma;
   if (can_stream) return kRegimeStream;
   return generic;
@@ -205,6 +212,12 @@ static cudaError_t launch_main(const KArgs& a, int dtype, const DeviceInfo& di, 
   const Regime reg = pick_regime(a, dtype, di.smem_optin);
   if (reg == kRegimeTma) return launch_tma(a, dtype, di.num_sms, di.smem_optin, stream);
   if (reg == kRegimeStream) return launch_stream(a, dtype, di.num_sms, stream);
+  if (reg == kRegimeCluster) {
+    const cudaError_t e = launch_cluster_single(a, dtype, di.smem_optin, stream);
+    if (e != cudaSuccess || !a.fused_finalize) return e;
+    finalize_kernel<<<1, 1024, 0, stream>>>(a);   // this kernel leaves the final reduction to a launch of its own
+    return cudaGetLastError();
+  }
   return launch_generic(a, dtype, reg == kRegimeWarp, rows_vectorizable(a, dtype), di.num_sms, stream);
 }
 
@@ -459,6 +472,7 @@ const char* codistill_kernel_regime(int n, int64_t rows, int64_t classes, int64_
     case kRegimeWarp: return "warp";
     case kRegimeBlock: return "block";
     case kRegimeStream: return "stream";
+    case kRegimeCluster: return "cluster";
     default: return "tma";
   }
 }

@@ -18,10 +18,12 @@
 //   d/dz_ic of T^2 sum_{j != i} KL(..)   = T (n t_ic - Q_c)
 // so again one read of the n rows per pass serves all n models; pass A adds sum_c exp((z - m) / T).
 #include <math.h>
+#include <stdlib.h>
 #include <string.h>
 
 #include <type_traits>
 
+#include "cluster_args.cuh"
 #include "stream_common.cuh"
 
 namespace codistill {
@@ -638,9 +640,10 @@ extern "C" int codistill_loss_fwd_bwd_all(const codistill_all_params_t* p, void*
   const AllLayout l = all_layout(p->n, p->rows);
   if (p->workspace_bytes < l.total) return CODISTILL_ERR_WORKSPACE;
 
-  int dev = 0, num_sms = 0;
+  int dev = 0, num_sms = 0, smem_optin = 0;
   if (cudaGetDevice(&dev) != cudaSuccess) return CODISTILL_ERR_CUDA;
   if (cudaDeviceGetAttribute(&num_sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) return CODISTILL_ERR_CUDA;
+  if (cudaDeviceGetAttribute(&smem_optin, cudaDevAttrMaxSharedMemoryPerBlockOptin, dev) != cudaSuccess) return CODISTILL_ERR_CUDA;
 
   char* ws = static_cast<char*>(p->workspace);
   AllArgs a;
@@ -669,7 +672,38 @@ extern "C" int codistill_loss_fwd_bwd_all(const codistill_all_params_t* p, void*
   if (launch_prep_rows(a.hdr, const_cast<int64_t*>(a.partials), a.labels, a.mask, a.rows, a.classes, stream) != cudaSuccess)
     return CODISTILL_ERR_CUDA;
   if (a.rows > 0) {
-    const cudaError_t e = p->dtype == CODISTILL_F32 ? all_launch<float>(a, num_sms, stream) : all_launch<__nv_bfloat16>(a, num_sms, stream);
+    // Long rows: the cluster-resident kernel reads every logit from HBM once (the n row images of a row
+    // index stay in the shared memory of a cluster); the direct-load kernel above reads them twice.
+    // CODISTILL_REGIME=stream keeps the direct-load kernel (for measurements).
+    const char* want = getenv("CODISTILL_REGIME");
+    const bool keep_direct = want != nullptr && strcmp(want, "stream") == 0;
+    cudaError_t e;
+    if (!keep_direct && cluster_fits(p->n, p->classes, p->row_stride, p->dtype, smem_optin)) {
+      ClArgs c;
+      memset(&c, 0, sizeof(c));
+      for (int i = 0; i < p->n; ++i) { c.model[i] = a.model[i]; c.grad[i] = a.grad[i]; }
+      c.labels = a.labels;
+      c.mask = a.mask;
+      c.row_loss = a.row_loss;
+      c.row_flags = a.row_flags;
+      c.hdr = a.hdr;
+      c.partials = a.partials;
+      c.rows_total = a.rows;
+      c.row_begin = 0;
+      c.row_end = a.rows;
+      c.classes = a.classes;
+      c.row_stride = a.row_stride;
+      c.n = a.n;
+      c.pairwise = a.peer_reduce == CODISTILL_PEERS_PAIRWISE_MEAN;
+      c.reduction = a.reduction;
+      c.centred = a.centred;
+      c.alpha = a.alpha;
+      c.eps = a.eps;
+      c.temperature = p->dist_kind == CODISTILL_DIST_KL_SOFTMAX ? p->temperature : 1.f;
+      e = launch_cluster(c, p->dtype, p->dist_kind == CODISTILL_DIST_KL_SOFTMAX ? kClKlPairwise : kClMse, true, smem_optin, stream);
+    } else {
+      e = p->dtype == CODISTILL_F32 ? all_launch<float>(a, num_sms, stream) : all_launch<__nv_bfloat16>(a, num_sms, stream);
+    }
     if (e != cudaSuccess) return CODISTILL_ERR_CUDA;
   }
   finalize_all_kernel<<<a.n, 1024, 0, stream>>>(a);

@@ -1,0 +1,844 @@
+// Cluster-resident kernel for long rows ("cluster" regime): every logit is read from HBM once.
+//
+// A thread-block cluster of K CTAs works on one row index at a time.  CTA k of the cluster owns a
+// fixed range of the 16-byte segments of the row image and keeps that range of ALL n logit tensors
+// (the n codistilled models of Algorithm 1: own + peers) in its shared memory, brought in by 1-D bulk
+// asynchronous copies (cp.async.bulk, no multicast) that complete on one mbarrier.  Both passes then
+// run from shared memory:
+//   pass A  per tensor the online softmax statistics of the CTA's range (maximum with its first
+//           column, sum exp, sum z, and for the KL form sum exp at temperature T); the K partial
+//           results of a tensor are exchanged through distributed shared memory after one cluster
+//           barrier, so that every CTA knows the statistics of the whole row;
+//   pass B  column by column over the CTA's range with the n models side by side: distance terms
+//           and the gradient of every requested model, written with 16-byte stores.
+// The distance partial sums of a row are collected by CTA 0 of the cluster behind the next row's
+// cluster barrier (nobody waits for them), which then writes the row's loss and flag word.
+//
+// Served: the all-models call (model i against the other n-1, all i) and the single-model call
+// (model 0 against its peers) with the distances whose gradient needs row statistics of the peers:
+// MSE on centred logits and the softmax-KL form, and plain MSE as an option.  The arithmetic is the
+// one of rows_all.cu: per column the n logits are centred on their mean over the models,
+//   z_i - zbar_(-i) = n/(n-1) z'_i,   sum_{j != i} (z_i - z_j)^2 = n z'_i^2 + sum_j z'_j^2,
+// and for KL with t_j = softmax(z_j / T), Q = sum_j t_j, E = sum_j t_j log t_j,
+//   sum_{j != i} KL(t_j || t_i) = sum_c (E_c - Q_c log t_ic),   d/dz_ic = T (n t_ic - Q_c) / ... .
+// A single-model call is the i = 0 part of the same sums.  The KL distance to the softmax of the
+// averaged peer logits (mean target, single-model call only) takes the statistics of that average
+// as one more tensor in pass A.
+#include <cooperative_groups.h>
+#include <stdlib.h>
+#include <string.h>
+
+#include <map>
+#include <mutex>
+#include <tuple>
+#include <type_traits>
+
+#include "bulk_copy.cuh"
+#include "cluster_args.cuh"
+#include "common.cuh"
+#include "seg_math.cuh"
+
+namespace cg = cooperative_groups;
+
+namespace codistill {
+
+constexpr int kClThreads = 256;
+constexpr int kClWarps = kClThreads / 32;
+constexpr int kClMaxRecs = 3;                      // pass-A records per warp (its range spans at most that many tensors)
+constexpr int kClMaxCluster = 16;
+constexpr int kClCtrlBytes = 4096;
+constexpr uint32_t kClCopyPiece = 32768;
+constexpr unsigned long long kClWaitLimitNs = 2000000000ull;   // bounded waits: 2 s, then CODISTILL_DEV_TIMEOUT
+
+// what one warp found in a sub-range of one tensor
+struct ClRec { float m; int seg; float S, sum_z, S_T; int tensor; };
+// what one CTA found in its range of one tensor
+struct ClPart { float m; int col; float S, sum_z, S_T, zy; int has_y; int pad; };
+// statistics of a whole row of one tensor
+struct ClStat { float m, S, sum_z, S_T, zy; int col; };
+
+struct ClCtrl {
+  uint64_t full;                           // bulk copies of the current row have landed
+  int abort_flag;
+  int nrec[kClWarps];
+  ClRec rec[kClWarps][kClMaxRecs];
+  ClRec rec_mean[kClWarps];                // KL mean target: statistics of the averaged peers
+  ClPart part[2][kClMax + 1];              // [row parity][tensor]; slot n: the averaged peers
+  float dpart[2][kClMax + 1];              // distance partial sums per model; slot kClMax: sum_j z'_j^2
+  float dwarp[kClWarps][kClMax + 1];
+  ClStat stat[kClMax + 1];                 // current row, combined over the cluster
+  ClStat pend[2][kClMax + 1];              // CTA 0: statistics of the rows whose loss is still to be written
+  long long pend_row[2];
+  int pend_y[2];
+};
+static_assert(sizeof(ClCtrl) <= kClCtrlBytes, "control block fits its slot");
+
+// Wait for a phase of the copy barrier, but never for ever: after the limit the CTA-wide abort flag and the
+// device status are set and later waits return early (results are then invalid, control flow stays uniform).
+__device__ __noinline__ void cl_wait_slow(uint64_t* bar, uint32_t parity, ClCtrl* ctrl, WsHeader* hdr, bool heed_abort) {
+  volatile int* abort_flag = &ctrl->abort_flag;
+  uint32_t polls = 0;
+  unsigned long long t0 = 0;
+  while (!mbar_try_wait(bar, parity)) {
+    if ((++polls & 0x3FFu) == 0) {
+      if (heed_abort && *abort_flag) return;
+      const unsigned long long now = global_timer_ns();
+      if (t0 == 0) {
+        t0 = now;
+      } else if (now - t0 > kClWaitLimitNs) {
+        *abort_flag = 1;
+        atomicOr(&hdr->status, CODISTILL_DEV_TIMEOUT);
+        return;
+      }
+    }
+  }
+}
+__device__ __forceinline__ void cl_wait(uint64_t* bar, uint32_t parity, ClCtrl* ctrl, WsHeader* hdr) {
+  if (mbar_try_wait(bar, parity)) return;
+  cl_wait_slow(bar, parity, ctrl, hdr, true);
+}
+
+// exp((z - m) / T) for a pair of columns; l2eT = log2(e) / T
+template <typename T>
+__device__ __forceinline__ float2 exp_temp2(float2 z, float m, float inv_T, float l2eT) {
+  if constexpr (sizeof(T) == 4) {
+    return make_float2(expf((z.x - m) * inv_T), expf((z.y - m) * inv_T));
+  } else {
+    const float2 t = __ffma2_rn(z, make_float2(l2eT, l2eT), make_float2(-m * l2eT, -m * l2eT));
+    return make_float2(ex2_approx(t.x), ex2_approx(t.y));
+  }
+}
+// exp(x), x in natural units: full precision for fp32 logits, the hardware exp2 for bf16 logits
+template <typename T>
+__device__ __forceinline__ float exp_nat1(float x) {
+  if constexpr (sizeof(T) == 4) return expf(x); else return ex2_approx(x * kLog2e);
+}
+
+// Running statistics of one thread over its segments of one tensor (visited in rising order).
+struct ClAcc {
+  float best;       // finite start value, so that the first rescale is exp2(-huge) = 0 and never NaN
+  int best_seg;
+  float2 s2, t2, zs2;
+  __device__ void reset() { best = -3.0e38f; best_seg = 0x7fffffff; s2 = make_float2(0.f, 0.f); t2 = s2; zs2 = s2; }
+};
+
+template <typename T, bool TEMP>
+__device__ __forceinline__ void cl_raise(ClAcc& acc, float fm, int s, float inv_T) {
+  if (fm > acc.best) {
+    const float sc = rescale_exp2<T>((acc.best - fm) * kLog2e);
+    acc.s2 = __fmul2_rn(acc.s2, make_float2(sc, sc));
+    if constexpr (TEMP) {
+      const float st = rescale_exp2<T>((acc.best - fm) * (kLog2e * inv_T));
+      acc.t2 = __fmul2_rn(acc.t2, make_float2(st, st));
+    }
+    acc.best = fm;
+    acc.best_seg = s;
+  }
+}
+
+// one whole segment (all of its columns lie inside the row)
+template <typename T, bool TEMP>
+__device__ __forceinline__ void cl_sweep_seg(ClAcc& acc, const uint4& raw, int s, float inv_T) {
+  constexpr int H = SegOps<T>::H;
+  cl_raise<T, TEMP>(acc, SegOps<T>::to_float(SegOps<T>::fold(raw)), s, inv_T);
+  const float2 l2e2 = make_float2(kLog2e, kLog2e);
+  const float2 nmk = make_float2(-acc.best * kLog2e, -acc.best * kLog2e);
+  float2 z2[H];
+  SegOps<T>::unpack2(raw, z2);
+#pragma unroll
+  for (int h = 0; h < H; ++h) {
+    acc.s2 = __fadd2_rn(acc.s2, exp_shift2<T>(z2[h], acc.best, l2e2, nmk));
+    acc.zs2 = __fadd2_rn(acc.zs2, z2[h]);
+    if constexpr (TEMP) acc.t2 = __fadd2_rn(acc.t2, exp_temp2<T>(z2[h], acc.best, inv_T, kLog2e * inv_T));
+  }
+}
+
+// a ragged segment (first or last of the row image): only the columns inside the row count
+template <typename T, bool TEMP>
+__device__ __noinline__ void cl_sweep_edge(ClAcc& acc, uint4 raw, int s, int head, int64_t C, float inv_T) {
+  constexpr int V = SegOps<T>::V;
+  float z[V];
+  SegOps<T>::unpack(raw, z);
+  float fm = -3.0e38f;
+#pragma unroll
+  for (int e = 0; e < V; ++e) {
+    const int64_t c = (int64_t)s * V - head + e;
+    if (c >= 0 && c < C) fm = fmaxf(fm, z[e]);
+  }
+  cl_raise<T, TEMP>(acc, fm, s, inv_T);
+  const float2 l2e2 = make_float2(kLog2e, kLog2e);
+  const float2 nmk = make_float2(-acc.best * kLog2e, -acc.best * kLog2e);
+#pragma unroll
+  for (int e = 0; e < V; ++e) {
+    const int64_t c = (int64_t)s * V - head + e;
+    if (c >= 0 && c < C) {
+      acc.s2.x += exp_shift2<T>(make_float2(z[e], z[e]), acc.best, l2e2, nmk).x;
+      acc.zs2.x += z[e];
+      if constexpr (TEMP) acc.t2.x += exp_temp2<T>(make_float2(z[e], z[e]), acc.best, inv_T, kLog2e * inv_T).x;
+    }
+  }
+}
+
+// Reduces the lanes' accumulators of one sub-range to one record (all lanes take part).
+template <typename T, bool TEMP>
+__device__ __forceinline__ ClRec cl_warp_record(const ClAcc& acc, int tensor, float inv_T) {
+  const unsigned key = float_order_key(acc.best + 0.f);   // -0 is folded onto +0: they tie
+  const unsigned key_w = __reduce_max_sync(0xffffffffu, key);
+  ClRec r;
+  r.seg = (int)__reduce_min_sync(0xffffffffu, key == key_w ? (unsigned)acc.best_seg : 0x7fffffffu);
+  r.m = float_from_order_key(key_w);
+  r.S = warp_sum((acc.s2.x + acc.s2.y) * rescale_exp2<T>((acc.best - r.m) * kLog2e));
+  r.sum_z = warp_sum(acc.zs2.x + acc.zs2.y);
+  r.S_T = 0.f;
+  if constexpr (TEMP) r.S_T = warp_sum((acc.t2.x + acc.t2.y) * rescale_exp2<T>((acc.best - r.m) * (kLog2e * inv_T)));
+  r.tensor = tensor;
+  return r;
+}
+
+// ------------------------------------------------------------------ the kernel
+// T: element type; N: resident tensors; MODE: ClMode; ALL: every model's outputs (else model 0's only).
+template <typename T, int N, int MODE, bool ALL>
+__global__ void __launch_bounds__(kClThreads, 2) rows_cluster_kernel(const __grid_constant__ ClArgs a) {
+  constexpr int V = SegOps<T>::V;
+  constexpr int H = SegOps<T>::H;
+  constexpr int ES = (int)sizeof(T);
+  constexpr bool KL = MODE != kClMse;
+  constexpr bool KLM = MODE == kClKlMeanTarget;
+  constexpr int NOUT = ALL ? N : 1;
+  constexpr int NSTAT = KLM ? N + 1 : N;
+  constexpr int NW = kClWarps, NT = kClThreads;
+  static_assert(!(KLM && ALL), "the mean-target KL distance is a single-model form");
+  static_assert(N >= 2 && N <= kClMax, "tensor count");
+  extern __shared__ __align__(128) unsigned char smem_raw[];
+  ClCtrl* ctrl = reinterpret_cast<ClCtrl*>(smem_raw);
+  char* slices = reinterpret_cast<char*>(smem_raw) + kClCtrlBytes;
+  cg::cluster_group cluster = cg::this_cluster();
+  const int K = (int)cluster.num_blocks();
+  const int rank = (int)cluster.block_rank();
+  const int cid = (int)(blockIdx.x / K), ncl = (int)(gridDim.x / K);
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  const int64_t C = a.classes, R = a.rows_total;
+  const float inv_C = 1.f / (float)C;
+  const float inv_T = KL ? 1.f / a.temperature : 1.f;
+  const bool t_one = !KL || a.temperature == 1.f;
+
+  if (tid == 0) {
+    mbar_init(&ctrl->full, 1);
+    ctrl->abort_flag = 0;
+    mbar_init_fence();
+  }
+  wait_for_prior_grid();  // from here on the workspace header and the valid-row counts are read
+  __syncthreads();
+
+  float w = 1.f;
+  if (a.reduction == CODISTILL_REDUCE_MEAN_VALID) {
+    const int nb = a.hdr->prep_blocks;
+    int64_t nv = 0;
+    for (int b = 0; b < nb; ++b) nv += a.partials[2 * b];
+    w = 1.f / (float)(nv > 1 ? nv : 1);
+  }
+  constexpr float kRatio = (float)N / (float)(N - 1);                 // z_i - zbar_(-i) = kRatio * z'_i
+  const float cd = w * a.alpha * (2.f * inv_C) * kRatio;               // z'_i -> w alpha dD_i/dz_i      (MSE)
+  const float cq = w * a.eps * inv_C;
+  const float cy = w * (1.f - a.eps);
+  const float ckl = KLM ? w * a.alpha * a.temperature                  // (p^T - t) -> w alpha dD/dz
+                        : w * a.alpha * a.temperature / (float)(N - 1);  // (n t_i - Q) -> w alpha dD_i/dz_i
+  const int seg_begin = rank * a.spc;
+
+  auto row_is_valid = [&](long long r) {
+    if (a.mask != nullptr && a.mask[r] == 0) return false;
+    const int32_t y = a.labels[r];
+    return y >= 0 && (int64_t)y < C;
+  };
+  // Thread 0: start the bulk copies of this CTA's range of row r for all n tensors.
+  auto issue_row = [&](long long r) {
+    const int64_t lr = r - a.row_begin;
+    const RowGeom g = row_geom<T>(lr, a.row_stride, C);
+    const int seg_end = min(seg_begin + a.spc, g.n_seg);
+    if (seg_end <= seg_begin) { mbar_arrive(&ctrl->full); return; }
+    const uint32_t begin = (uint32_t)seg_begin * 16u, end = (uint32_t)seg_end * 16u;
+    // The last row of the whole call may end inside a segment that reaches past the tensor: that
+    // segment is fetched element by element, whole-segment copies stop before it.
+    const uint32_t valid_end = (uint32_t)(g.head + C) * ES;
+    const bool clip = (r == R - 1) && ((a.row_stride - C) * ES < 16) && (valid_end & 15u) && end > (valid_end & ~15u);
+    const uint32_t copy_end = clip ? (valid_end & ~15u) : end;
+    const uint32_t bytes = copy_end > begin ? copy_end - begin : 0u;
+    const int64_t img_off = (lr * a.row_stride - g.head) * ES;   // image start relative to the tensor
+    if (clip) {
+#pragma unroll 1
+      for (int i = 0; i < N; ++i) {
+        const char* src = reinterpret_cast<const char*>(a.model[i]) + img_off;
+        char* dst = slices + (size_t)i * a.slice_bytes - begin;
+        for (uint32_t o = copy_end > begin ? copy_end : begin; o < valid_end; o += ES)
+          *reinterpret_cast<T*>(dst + o) = *reinterpret_cast<const T*>(src + o);
+      }
+    }
+    mbar_arrive_expect_tx(&ctrl->full, bytes * (uint32_t)N);
+#pragma unroll 1
+    for (int i = 0; i < N; ++i) {
+      const char* src = reinterpret_cast<const char*>(a.model[i]) + img_off + begin;
+      char* dst = slices + (size_t)i * a.slice_bytes;
+      for (uint32_t o = 0; o < bytes; o += kClCopyPiece)
+        bulk_g2s(dst + o, src + o, bytes - o < kClCopyPiece ? bytes - o : kClCopyPiece, &ctrl->full);
+    }
+  };
+  // CTA 0: loss and flag word of the pending row with parity `pp`, from the K distance partials.
+  auto finish_row = [&](int pp) {
+    for (int i = warp; i < NOUT; i += NW) {
+      float dv = 0.f, qv = 0.f;
+      if (lane < K) {
+        const float* dp = cluster.map_shared_rank(&ctrl->dpart[pp][0], lane);
+        dv = dp[i];
+        qv = dp[kClMax];
+      }
+      const float dsum = warp_sum(dv), qsum = warp_sum(qv);
+      if (lane == 0) {
+        const ClStat st = ctrl->pend[pp][i];
+        const long long r = ctrl->pend_row[pp];
+        const int y = ctrl->pend_y[pp];
+        const float ce = (st.m + logf(st.S)) - (1.f - a.eps) * st.zy - (a.eps * inv_C) * st.sum_z;
+        float D;
+        if constexpr (KLM) D = a.temperature * a.temperature * dsum;
+        else if constexpr (KL) D = a.temperature * a.temperature * dsum / (float)(N - 1);
+        else D = a.pairwise ? fmaf((float)N, dsum, qsum) * inv_C / (float)(N - 1) : dsum * kRatio * kRatio * inv_C;
+        uint32_t flags = (st.col == y) ? 1u : 0u;
+        int bit = 1;
+        for (int j = 0; j < N; ++j) {
+          if (j == i) continue;
+          if (ctrl->pend[pp][j].col == st.col) flags |= (1u << bit);
+          ++bit;
+        }
+        a.row_loss[(int64_t)i * R + r] = a.alpha != 0.f ? fmaf(a.alpha, D, ce) : ce;
+        a.row_flags[(int64_t)i * R + r] = flags;
+      }
+    }
+  };
+
+  int v = 0;                   // valid rows done by this cluster
+  long long issued = -1;       // thread 0: row whose copies were started last
+  for (long long r = a.row_begin + cid; r < a.row_end; r += ncl) {
+    const int64_t lr = r - a.row_begin;
+    const RowGeom g = row_geom<T>(lr, a.row_stride, C);
+    const int seg_end = min(seg_begin + a.spc, g.n_seg);
+    const int nseg = seg_end > seg_begin ? seg_end - seg_begin : 0;     // segments of this CTA's range in this row
+    const int64_t img_off = (lr * a.row_stride - g.head) * ES;
+    const int y = a.labels[r];
+    const bool valid = (a.mask == nullptr || a.mask[r] != 0) && y >= 0 && (int64_t)y < C;
+
+    if (!valid) {  // masked row: zero gradient rows, no loss, no counts; nothing is read
+#pragma unroll 1
+      for (int i = 0; i < NOUT; ++i) {
+        if (a.grad[i] == nullptr) continue;
+        char* g_img = reinterpret_cast<char*>(a.grad[i]) + img_off;
+        for (int q = tid; q < nseg; q += NT) {
+          const int s = seg_begin + q;
+          if (s >= g.seg_lo && s < g.seg_hi) {
+            *reinterpret_cast<uint4*>(g_img + (size_t)s * 16) = make_uint4(0u, 0u, 0u, 0u);
+          } else {
+#pragma unroll
+            for (int e = 0; e < V; ++e) {
+              const int64_t c = (int64_t)s * V - g.head + e;
+              if (c >= 0 && c < C) reinterpret_cast<T*>(g_img + (size_t)s * 16)[e] = Elem<T>::from_f32(0.f);
+            }
+          }
+        }
+      }
+      if (rank == 0 && tid < NOUT) { a.row_loss[(int64_t)tid * R + r] = 0.f; a.row_flags[(int64_t)tid * R + r] = 0u; }
+      continue;
+    }
+    const int par = v & 1;
+    if (tid == 0 && issued != r) { issue_row(r); issued = r; }
+    cl_wait(&ctrl->full, (uint32_t)v & 1u, ctrl, a.hdr);
+
+    // ================= pass A: statistics of this CTA's range, tensor by tensor
+    // The n * nseg (tensor, segment) items are dealt to the warps in equal contiguous shares, so a
+    // warp reduces once per tensor its share touches (at most kClMaxRecs times), not once per tensor.
+    {
+      const int total = N * nseg;
+      int lo = (int)(((long long)warp * total) / NW);
+      const int hi = (int)(((long long)(warp + 1) * total) / NW);
+      int nrec = 0;
+      while (lo < hi) {
+        const int i = lo / nseg;
+        const int q0 = lo - i * nseg;
+        const int q1 = min(hi - i * nseg, nseg);
+        const char* sl = slices + (size_t)i * a.slice_bytes;
+        ClAcc acc;
+        acc.reset();
+        for (int q = q0 + lane; q < q1; q += 32) {
+          const int s = seg_begin + q;
+          const uint4 raw = *reinterpret_cast<const uint4*>(sl + (size_t)q * 16);
+          if (s >= g.seg_lo && s < g.seg_hi) {
+            if (t_one) cl_sweep_seg<T, false>(acc, raw, s, inv_T); else cl_sweep_seg<T, KL>(acc, raw, s, inv_T);
+          } else {
+            if (t_one) cl_sweep_edge<T, false>(acc, raw, s, g.head, C, inv_T); else cl_sweep_edge<T, KL>(acc, raw, s, g.head, C, inv_T);
+          }
+        }
+        const ClRec rec = t_one ? cl_warp_record<T, false>(acc, i, inv_T) : cl_warp_record<T, KL>(acc, i, inv_T);
+        if (lane == 0 && nrec < kClMaxRecs) ctrl->rec[warp][nrec] = rec;
+        ++nrec;
+        lo = i * nseg + q1;
+      }
+      if (lane == 0) ctrl->nrec[warp] = nrec < kClMaxRecs ? nrec : kClMaxRecs;
+    }
+    if constexpr (KLM) {
+      // statistics of the averaged peer logits zbar = mean_{j >= 1} z_j at temperature T
+      ClAcc acc;
+      acc.reset();
+      const float inv_P = 1.f / (float)(N - 1);
+      for (int q = tid; q < nseg; q += NT) {
+        const int s = seg_begin + q;
+        float2 zb[H];
+#pragma unroll
+        for (int h = 0; h < H; ++h) zb[h] = make_float2(0.f, 0.f);
+#pragma unroll
+        for (int j = 1; j < N; ++j) {
+          float2 v2[H];
+          SegOps<T>::unpack2(*reinterpret_cast<const uint4*>(slices + (size_t)j * a.slice_bytes + (size_t)q * 16), v2);
+#pragma unroll
+          for (int h = 0; h < H; ++h) zb[h] = __fadd2_rn(zb[h], v2[h]);
+        }
+        float fm = -3.0e38f;
+        bool in[V];
+#pragma unroll
+        for (int e = 0; e < V; ++e) {
+          const int64_t c = (int64_t)s * V - g.head + e;
+          in[e] = c >= 0 && c < C;
+        }
+#pragma unroll
+        for (int h = 0; h < H; ++h) {
+          zb[h] = __fmul2_rn(zb[h], make_float2(inv_P, inv_P));
+          if (in[2 * h]) fm = fmaxf(fm, zb[h].x);
+          if (in[2 * h + 1]) fm = fmaxf(fm, zb[h].y);
+        }
+        cl_raise<T, true>(acc, fm, s, inv_T);
+#pragma unroll
+        for (int h = 0; h < H; ++h) {
+          const float2 e2 = exp_temp2<T>(zb[h], acc.best, inv_T, kLog2e * inv_T);
+          if (in[2 * h]) acc.t2.x += e2.x;
+          if (in[2 * h + 1]) acc.t2.y += e2.y;
+        }
+      }
+      const ClRec rec = cl_warp_record<T, true>(acc, N, inv_T);
+      if (lane == 0) ctrl->rec_mean[warp] = rec;
+    }
+    __syncthreads();
+    if (tid < NSTAT) {
+      // this CTA's partial result of tensor `tid`: records in rising segment order, a strictly larger
+      // maximum replaces the earlier one, so the first segment that attains the maximum is kept
+      float m = -3.0e38f, S = 0.f, sum_z = 0.f, S_T = 0.f;
+      int seg = 0x7fffffff;
+      auto take = [&](const ClRec& rc) {
+        const float mn = fmaxf(m, rc.m);
+        const float f_old = rescale_exp2<T>((m - mn) * kLog2e), f_new = rescale_exp2<T>((rc.m - mn) * kLog2e);
+        S = S * f_old + rc.S * f_new;
+        if (!t_one || tid == N) {   // the averaged peers (slot N) carry the tempered sum only
+          S_T = S_T * rescale_exp2<T>((m - mn) * (kLog2e * inv_T)) + rc.S_T * rescale_exp2<T>((rc.m - mn) * (kLog2e * inv_T));
+        }
+        sum_z += rc.sum_z;
+        if (rc.m > m) seg = rc.seg;
+        m = mn;
+      };
+      if (tid < N) {
+        for (int wv = 0; wv < NW; ++wv)
+          for (int k = 0; k < ctrl->nrec[wv]; ++k)
+            if (ctrl->rec[wv][k].tensor == tid) take(ctrl->rec[wv][k]);
+      } else {
+        for (int wv = 0; wv < NW; ++wv) take(ctrl->rec_mean[wv]);
+      }
+      ClPart p;
+      p.m = m; p.S = S; p.sum_z = sum_z; p.S_T = S_T; p.col = 0x7fffffff; p.zy = 0.f; p.has_y = 0; p.pad = 0;
+      if (tid < N) {
+        const T* sl = reinterpret_cast<const T*>(slices + (size_t)tid * a.slice_bytes);
+        if (seg >= seg_begin && seg < seg_end) {   // first column of that segment that attains the maximum
+#pragma unroll
+          for (int e = V - 1; e >= 0; --e) {
+            const int64_t c = (int64_t)seg * V - g.head + e;
+            if (c >= 0 && c < C && Elem<T>::to_f32(sl[(size_t)(seg - seg_begin) * V + e]) == m) p.col = (int)c;
+          }
+        }
+        const int seg_y = (g.head + y) / V;
+        if (seg_y >= seg_begin && seg_y < seg_end) {
+          p.zy = Elem<T>::to_f32(sl[(size_t)(seg_y - seg_begin) * V + (g.head + y) % V]);
+          p.has_y = 1;
+        }
+      }
+      ctrl->part[par][tid] = p;
+    }
+    cluster.sync();   // every CTA's partial results of this row are written (and its work on the previous row is done)
+
+    // ================= statistics of the whole row: warp i combines the K partial results of tensor i
+    for (int i = warp; i < NSTAT; i += NW) {
+      ClPart p;
+      p.m = -3.0e38f; p.col = 0x7fffffff; p.S = 0.f; p.sum_z = 0.f; p.S_T = 0.f; p.zy = 0.f; p.has_y = 0; p.pad = 0;
+      if (lane < K) p = *cluster.map_shared_rank(&ctrl->part[par][i], lane);
+      const unsigned key = float_order_key(p.m + 0.f);
+      const unsigned key_m = __reduce_max_sync(0xffffffffu, key);
+      const float m = float_from_order_key(key_m);
+      ClStat st;
+      st.m = m;
+      st.col = (int)__reduce_min_sync(0xffffffffu, key == key_m ? (unsigned)p.col : 0x7fffffffu);
+      st.S = warp_sum(p.S * rescale_exp2<T>((p.m - m) * kLog2e));
+      st.S_T = (t_one && i < N) ? st.S : warp_sum(p.S_T * rescale_exp2<T>((p.m - m) * (kLog2e * inv_T)));
+      st.sum_z = warp_sum(p.sum_z);
+      st.zy = warp_sum(p.has_y ? p.zy : 0.f);
+      if (lane == 0) ctrl->stat[i] = st;
+    }
+    if (rank == 0 && v >= 1) finish_row(par ^ 1);   // the previous valid row: all its distance partials are in
+    __syncthreads();
+    if (rank == 0 && tid < NSTAT) {
+      ctrl->pend[par][tid] = ctrl->stat[tid];
+      if (tid == 0) { ctrl->pend_row[par] = r; ctrl->pend_y[par] = y; }
+    }
+    float mi[N], cpi[N], cmi[N];                       // per model: maximum, w / S, class mean removed before the distance
+    float cti[KL ? NSTAT : 1], lsi[KL ? NSTAT : 1];    // KL: 1 / S_T and log S_T
+#pragma unroll
+    for (int i = 0; i < N; ++i) {
+      const ClStat st = ctrl->stat[i];
+      mi[i] = st.m;
+      cpi[i] = w * __frcp_rn(st.S);
+      cmi[i] = a.centred ? st.sum_z * inv_C : 0.f;
+      if constexpr (KL) { cti[i] = __frcp_rn(st.S_T); lsi[i] = logf(st.S_T); }
+    }
+    float mb = 0.f;   // KL mean target: maximum of the averaged peers
+    if constexpr (KLM) { const ClStat st = ctrl->stat[N]; mb = st.m; cti[N] = __frcp_rn(st.S_T); lsi[N] = logf(st.S_T); }
+
+    // ================= pass B: distance terms and gradients, the n models side by side
+    float2 dist2[NOUT], qs2 = make_float2(0.f, 0.f);
+#pragma unroll
+    for (int i = 0; i < NOUT; ++i) dist2[i] = make_float2(0.f, 0.f);
+    // Two neighbouring columns c, c + 1 (first_in / second_in: inside the row); zc: the n models' logits.
+    // Returns the gradient pairs of the requested models; `lab` says that c or c + 1 may be the label column.
+    auto column2 = [&](bool ragged, const float2 (&zc)[N], float2 (&gc)[NOUT], int64_t c, bool lab, bool first_in, bool second_in) {
+      const bool kRagged = ragged;   // some column of the pair may lie outside the row
+      float2 ncq = make_float2(-cq, -cq);
+      if (lab) ncq = make_float2((c == (int64_t)y) ? -(cq + cy) : -cq, (c + 1 == (int64_t)y) ? -(cq + cy) : -cq);
+      const float2 in2 = make_float2(first_in ? 1.f : 0.f, second_in ? 1.f : 0.f);
+      auto inside = [&](float2 x) { return kRagged ? __fmul2_rn(x, in2) : x; };
+      if constexpr (MODE == kClMse) {
+        float2 zp[N], mu = make_float2(0.f, 0.f), q = make_float2(0.f, 0.f);
+#pragma unroll
+        for (int i = 0; i < N; ++i) { zp[i] = __fadd2_rn(zc[i], make_float2(-cmi[i], -cmi[i])); mu = __fadd2_rn(mu, zp[i]); }
+        mu = __fmul2_rn(mu, make_float2(-1.f / (float)N, -1.f / (float)N));
+#pragma unroll
+        for (int i = 0; i < N; ++i) {
+          zp[i] = inside(__fadd2_rn(zp[i], mu));
+          q = __ffma2_rn(zp[i], zp[i], q);
+        }
+#pragma unroll
+        for (int i = 0; i < NOUT; ++i) {
+          const float nm = -mi[i] * kLog2e;
+          const float2 e = exp_shift2<T>(zc[i], mi[i], make_float2(kLog2e, kLog2e), make_float2(nm, nm));
+          gc[i] = __ffma2_rn(e, make_float2(cpi[i], cpi[i]), __ffma2_rn(make_float2(cd, cd), zp[i], ncq));
+          dist2[i] = __ffma2_rn(zp[i], zp[i], dist2[i]);
+        }
+        qs2 = __fadd2_rn(qs2, q);
+      } else if constexpr (MODE == kClKlPairwise) {
+        float2 t[N], lt[N], Q = make_float2(0.f, 0.f), E = make_float2(0.f, 0.f);
+#pragma unroll
+        for (int i = 0; i < N; ++i) {
+          float2 e1 = make_float2(0.f, 0.f), et;
+          if (t_one || i < NOUT) {
+            const float nm = -mi[i] * kLog2e;
+            e1 = exp_shift2<T>(zc[i], mi[i], make_float2(kLog2e, kLog2e), make_float2(nm, nm));
+          }
+          et = t_one ? e1 : exp_temp2<T>(zc[i], mi[i], inv_T, kLog2e * inv_T);
+          t[i] = inside(__fmul2_rn(et, make_float2(cti[i], cti[i])));
+          const float2 x = __fadd2_rn(zc[i], make_float2(-mi[i], -mi[i]));
+          const float2 l = __ffma2_rn(x, make_float2(inv_T, inv_T), make_float2(-lsi[i], -lsi[i]));
+          lt[i] = make_float2(fmaxf(l.x, -3.0e38f), fmaxf(l.y, -3.0e38f));   // log t_i, kept finite: 0 * log 0 = 0
+          Q = __fadd2_rn(Q, t[i]);
+          E = __ffma2_rn(t[i], lt[i], E);
+          if (i < NOUT) gc[i] = __ffma2_rn(e1, make_float2(cpi[i], cpi[i]), ncq);
+        }
+        const float2 nQ = make_float2(-Q.x, -Q.y);
+#pragma unroll
+        for (int i = 0; i < NOUT; ++i) {
+          gc[i] = __ffma2_rn(make_float2(ckl, ckl), __ffma2_rn(make_float2((float)N, (float)N), t[i], nQ), gc[i]);
+          dist2[i] = __fadd2_rn(dist2[i], __ffma2_rn(nQ, lt[i], E));   // sum_{j != i} t_j (log t_j - log t_i)
+        }
+      } else {
+        // KL to the softmax of the averaged peers: t = softmax(zbar / T), p^T = softmax(z_0 / T)
+        const float inv_P = 1.f / (float)(N - 1);
+        float2 zb = make_float2(0.f, 0.f);
+#pragma unroll
+        for (int j = 1; j < N; ++j) zb = __fadd2_rn(zb, zc[j]);
+        zb = __fmul2_rn(zb, make_float2(inv_P, inv_P));
+        const float nm = -mi[0] * kLog2e;
+        const float2 e1 = exp_shift2<T>(zc[0], mi[0], make_float2(kLog2e, kLog2e), make_float2(nm, nm));
+        const float2 eT = t_one ? e1 : exp_temp2<T>(zc[0], mi[0], inv_T, kLog2e * inv_T);
+        const float2 pT = __fmul2_rn(eT, make_float2(cti[0], cti[0]));
+        const float2 x0 = __fadd2_rn(zc[0], make_float2(-mi[0], -mi[0]));
+        const float2 lp = __ffma2_rn(x0, make_float2(inv_T, inv_T), make_float2(-lsi[0], -lsi[0]));
+        const float2 tb = inside(__fmul2_rn(exp_temp2<T>(zb, mb, inv_T, kLog2e * inv_T), make_float2(cti[N], cti[N])));
+        const float2 xb = __fadd2_rn(zb, make_float2(-mb, -mb));
+        const float2 lb = __ffma2_rn(xb, make_float2(inv_T, inv_T), make_float2(-lsi[N], -lsi[N]));
+        const float2 dl = make_float2(fmaxf(lb.x, -3.0e38f) - fmaxf(lp.x, -3.0e38f), fmaxf(lb.y, -3.0e38f) - fmaxf(lp.y, -3.0e38f));
+        gc[0] = __ffma2_rn(make_float2(ckl, ckl), __fadd2_rn(pT, make_float2(-tb.x, -tb.y)), __ffma2_rn(e1, make_float2(cpi[0], cpi[0]), ncq));
+        dist2[0] = __ffma2_rn(tb, dl, dist2[0]);
+      }
+    };
+    const int seg_y = (g.head + y) / V;
+    for (int q = tid; q < nseg; q += NT) {
+      const int s = seg_begin + q;
+      const int64_t cbase = (int64_t)s * V - g.head;
+      const bool lab = s == seg_y;
+      uint4 rw[N];
+#pragma unroll
+      for (int i = 0; i < N; ++i) rw[i] = *reinterpret_cast<const uint4*>(slices + (size_t)i * a.slice_bytes + (size_t)q * 16);
+      if (s >= g.seg_lo && s < g.seg_hi) {
+#pragma unroll
+        for (int h = 0; h < H; ++h) {
+          float2 zc[N], gc[NOUT];
+#pragma unroll
+          for (int i = 0; i < N; ++i) {
+            if constexpr (ES == 4) {
+              zc[i] = h == 0 ? make_float2(__uint_as_float(rw[i].x), __uint_as_float(rw[i].y))
+                             : make_float2(__uint_as_float(rw[i].z), __uint_as_float(rw[i].w));
+            } else {
+              const uint32_t word = h == 0 ? rw[i].x : h == 1 ? rw[i].y : h == 2 ? rw[i].z : rw[i].w;
+              zc[i] = make_float2(__uint_as_float(word << 16), __uint_as_float(word & 0xFFFF0000u));
+            }
+          }
+          column2(false, zc, gc, cbase + 2 * h, lab, true, true);
+#pragma unroll
+          for (int i = 0; i < NOUT; ++i) {
+            if constexpr (ES == 4) {
+              if (h == 0) { rw[i].x = __float_as_uint(gc[i].x); rw[i].y = __float_as_uint(gc[i].y); }
+              else { rw[i].z = __float_as_uint(gc[i].x); rw[i].w = __float_as_uint(gc[i].y); }
+            } else {
+              const __nv_bfloat162 pk = __floats2bfloat162_rn(gc[i].x, gc[i].y);
+              const uint32_t word = *reinterpret_cast<const uint32_t*>(&pk);
+              if (h == 0) rw[i].x = word; else if (h == 1) rw[i].y = word; else if (h == 2) rw[i].z = word; else rw[i].w = word;
+            }
+          }
+        }
+#pragma unroll
+        for (int i = 0; i < NOUT; ++i)
+          if (a.grad[i] != nullptr) *reinterpret_cast<uint4*>(reinterpret_cast<char*>(a.grad[i]) + img_off + (size_t)s * 16) = rw[i];
+      } else {
+        // ragged segment: same arithmetic, columns outside the row contribute nothing and are not written
+#pragma unroll 1
+        for (int h = 0; h < H; ++h) {
+          float2 zc[N], gc[NOUT];
+          const int64_t c0 = cbase + 2 * h;
+          const bool in0 = c0 >= 0 && c0 < C, in1 = c0 + 1 >= 0 && c0 + 1 < C;
+#pragma unroll
+          for (int i = 0; i < N; ++i) {
+            const T* el = reinterpret_cast<const T*>(slices + (size_t)i * a.slice_bytes + (size_t)q * 16) + 2 * h;
+            zc[i] = make_float2(in0 ? Elem<T>::to_f32(el[0]) : mi[i], in1 ? Elem<T>::to_f32(el[1]) : mi[i]);
+          }
+          column2(true, zc, gc, c0, lab, in0, in1);
+#pragma unroll
+          for (int i = 0; i < NOUT; ++i) {
+            if (a.grad[i] == nullptr) continue;
+            T* ge = reinterpret_cast<T*>(reinterpret_cast<char*>(a.grad[i]) + img_off + (size_t)s * 16) + 2 * h;
+            if (in0) ge[0] = Elem<T>::from_f32(gc[i].x);
+            if (in1) ge[1] = Elem<T>::from_f32(gc[i].y);
+          }
+        }
+      }
+    }
+
+    // ================= distance partial sums of this CTA (read by CTA 0 behind the next cluster barrier)
+#pragma unroll
+    for (int i = 0; i < NOUT; ++i) {
+      const float dw = warp_sum(dist2[i].x + dist2[i].y);
+      if (lane == 0) ctrl->dwarp[warp][i] = dw;
+    }
+    if constexpr (MODE == kClMse) {
+      const float qw = warp_sum(qs2.x + qs2.y);
+      if (lane == 0) ctrl->dwarp[warp][kClMax] = qw;
+    }
+    __syncthreads();   // pass B has read the ranges: they may be overwritten; the warps' partial sums are in place
+    if (tid == 0) {
+      // start the copies of the next valid row of this cluster behind the arithmetic of other CTAs on this SM
+      long long r2 = r + ncl;
+      while (r2 < a.row_end && !row_is_valid(r2)) r2 += ncl;
+      if (r2 < a.row_end) { issue_row(r2); issued = r2; }
+    }
+    if (tid <= kClMax && (tid < NOUT || tid == kClMax)) {
+      float d = 0.f;
+      if (tid < NOUT || MODE == kClMse) {
+#pragma unroll
+        for (int wv = 0; wv < NW; ++wv) d += ctrl->dwarp[wv][tid];
+      }
+      ctrl->dpart[par][tid] = d;
+    }
+    ++v;
+  }
+
+  // ---------------- the last valid row's loss; nobody leaves while its shared memory may still be read
+  cluster.sync();
+  if (rank == 0 && v >= 1) finish_row((v - 1) & 1);
+  if (ctrl->abort_flag && tid == 0) {
+    // a wait ran out: give copies that may still be in flight one more bounded interval before the CTA ends
+    cl_wait_slow(&ctrl->full, (uint32_t)(v + 1) & 1u, ctrl, a.hdr, false);
+  }
+  cluster.sync();
+}
+
+// ------------------------------------------------------------------ host side
+struct ClPlan {
+  int cluster;           // CTAs per cluster (0: the kernel does not take the call)
+  int spc;
+  uint32_t slice_bytes;
+  uint32_t smem_bytes;
+};
+
+static int cluster_size_override() {
+  const char* s = getenv("CODISTILL_CLUSTER_SIZE");
+  if (s == nullptr) return 0;
+  const int k = atoi(s);
+  return (k == 1 || k == 2 || k == 4 || k == 8 || k == 16) ? k : 0;
+}
+
+// Smallest cluster whose CTAs keep their share of the n row images in about half an SM's shared
+// memory (two CTAs per SM: one computes while the other's copies are in flight).
+ClPlan cluster_plan(int n, int64_t classes, int64_t row_stride, int dtype, int smem_optin) {
+  ClPlan p = {0, 0, 0, 0};
+  if (n < 2 || n > kClMax) return p;
+  const int64_t n_seg = dtype == CODISTILL_F32 ? max_row_segments<float>(row_stride, classes)
+                                               : max_row_segments<__nv_bfloat16>(row_stride, classes);
+  if (n_seg * 16 < 8192 || classes > (int64_t)1 << 24) return p;
+  const int64_t half = ((int64_t)smem_optin + 1024) / 2 - 1024;
+  const int forced = cluster_size_override();
+  for (int k = forced ? forced : 1; k <= (forced ? forced : kClMaxCluster); k *= 2) {
+    const int64_t spc = (n_seg + k - 1) / k;
+    const int64_t slice = (spc * 16 + 127) & ~(int64_t)127;
+    const int64_t smem = kClCtrlBytes + (int64_t)n * slice;
+    if (smem <= (forced ? (int64_t)smem_optin : half)) {
+      p.cluster = k;
+      p.spc = (int)spc;
+      p.slice_bytes = (uint32_t)slice;
+      p.smem_bytes = (uint32_t)smem;
+      return p;
+    }
+  }
+  return p;
+}
+
+template <typename T, int N, int MODE, bool ALL>
+static cudaError_t cluster_launch_one(const ClArgs& a, const ClPlan& p, cudaStream_t stream) {
+  auto kernel = rows_cluster_kernel<T, N, MODE, ALL>;
+  // per kernel and launch shape: attributes set and the number of co-resident clusters asked once per device
+  static std::mutex mu;
+  static std::map<std::tuple<int, int, uint32_t>, int> known;
+  int dev = 0;
+  cudaError_t e = cudaGetDevice(&dev);
+  if (e != cudaSuccess) return e;
+  cudaLaunchConfig_t cfg = {};
+  cfg.blockDim = dim3(kClThreads);
+  cfg.dynamicSmemBytes = p.smem_bytes;
+  cfg.stream = stream;
+  cudaLaunchAttribute attr[2];
+  attr[0].id = cudaLaunchAttributeClusterDimension;
+  attr[0].val.clusterDim.x = (unsigned)p.cluster;
+  attr[0].val.clusterDim.y = 1;
+  attr[0].val.clusterDim.z = 1;
+  attr[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[1].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = 1;
+  int max_clusters = 0;
+  {
+    std::lock_guard<std::mutex> lock(mu);
+    const auto key = std::make_tuple(dev, p.cluster, p.smem_bytes);
+    const auto it = known.find(key);
+    if (it != known.end()) {
+      max_clusters = it->second;
+    } else {
+      if ((e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)p.smem_bytes)) != cudaSuccess) return e;
+      if (p.cluster > 8 && (e = cudaFuncSetAttribute(kernel, cudaFuncAttributeNonPortableClusterSizeAllowed, 1)) != cudaSuccess) return e;
+      cfg.gridDim = dim3((unsigned)p.cluster);
+      if ((e = cudaOccupancyMaxActiveClusters(&max_clusters, kernel, &cfg)) != cudaSuccess) return e;
+      if (max_clusters < 1) return cudaErrorLaunchOutOfResources;
+      known[key] = max_clusters;
+    }
+  }
+  const int64_t rows = a.row_end - a.row_begin;
+  const int64_t clusters = rows < max_clusters ? rows : max_clusters;
+  cfg.gridDim = dim3((unsigned)(clusters * p.cluster));
+  cfg.numAttrs = 2;
+  e = cudaLaunchKernelEx(&cfg, kernel, a);
+  return e != cudaSuccess ? e : cudaGetLastError();
+}
+
+template <typename T, int N>
+static cudaError_t cluster_launch_n(const ClArgs& a, const ClPlan& p, int mode, bool all, cudaStream_t stream) {
+  if (mode == kClMse) return all ? cluster_launch_one<T, N, kClMse, true>(a, p, stream) : cluster_launch_one<T, N, kClMse, false>(a, p, stream);
+  if (mode == kClKlPairwise)
+    return all ? cluster_launch_one<T, N, kClKlPairwise, true>(a, p, stream) : cluster_launch_one<T, N, kClKlPairwise, false>(a, p, stream);
+  return all ? cudaErrorNotSupported : cluster_launch_one<T, N, kClKlMeanTarget, false>(a, p, stream);
+}
+
+template <typename T>
+static cudaError_t cluster_launch_t(const ClArgs& a, const ClPlan& p, int mode, bool all, cudaStream_t stream) {
+  switch (a.n) {
+    case 2: return cluster_launch_n<T, 2>(a, p, mode, all, stream);
+    case 3: return cluster_launch_n<T, 3>(a, p, mode, all, stream);
+    case 4: return cluster_launch_n<T, 4>(a, p, mode, all, stream);
+    case 5: return cluster_launch_n<T, 5>(a, p, mode, all, stream);
+    case 6: return cluster_launch_n<T, 6>(a, p, mode, all, stream);
+    case 7: return cluster_launch_n<T, 7>(a, p, mode, all, stream);
+    case 8: return cluster_launch_n<T, 8>(a, p, mode, all, stream);
+    default: return cudaErrorNotSupported;
+  }
+}
+
+// Launches the cluster-resident kernel for rows [row_begin, row_end).  `mode`: ClMode; `all`: every model's outputs.
+cudaError_t launch_cluster(ClArgs a, int dtype, int mode, bool all, int smem_optin, cudaStream_t stream) {
+  const ClPlan p = cluster_plan(a.n, a.classes, a.row_stride, dtype, smem_optin);
+  if (p.cluster == 0) return cudaErrorNotSupported;
+  if (a.row_end <= a.row_begin) return cudaSuccess;
+  a.spc = p.spc;
+  a.slice_bytes = p.slice_bytes;
+  return dtype == CODISTILL_F32 ? cluster_launch_t<float>(a, p, mode, all, stream) : cluster_launch_t<__nv_bfloat16>(a, p, mode, all, stream);
+}
+
+bool cluster_fits(int n, int64_t classes, int64_t row_stride, int dtype, int smem_optin) {
+  return cluster_plan(n, classes, row_stride, dtype, smem_optin).cluster != 0;
+}
+
+// Whether the single-model call described by `a` can be served by the cluster-resident kernel.
+bool cluster_supported(const KArgs& a, int dtype, int smem_optin) {
+  if (a.n_peers < 1 || a.n_peers + 1 > kClMax) return false;
+  if (a.dist != CODISTILL_DIST_MSE_LOGITS && a.dist != CODISTILL_DIST_KL_SOFTMAX && a.dist != CODISTILL_DIST_MSE_CENTRED) return false;
+  uintptr_t bits = reinterpret_cast<uintptr_t>(a.own) | reinterpret_cast<uintptr_t>(a.grad);
+  for (int j = 0; j < a.n_peers; ++j) bits |= reinterpret_cast<uintptr_t>(a.peers[j]);
+  if (bits & 15u) return false;
+  return cluster_plan(a.n_peers + 1, a.classes, a.row_stride, dtype, smem_optin).cluster != 0;
+}
+
+// The single-model call on the cluster-resident kernel: own logits as model 0, the peers behind it.
+cudaError_t launch_cluster_single(const KArgs& k, int dtype, int smem_optin, cudaStream_t stream) {
+  ClArgs a;
+  memset(&a, 0, sizeof(a));
+  a.model[0] = k.own;
+  for (int j = 0; j < k.n_peers; ++j) a.model[1 + j] = k.peers[j];
+  a.grad[0] = k.grad;
+  a.labels = k.labels;
+  a.mask = k.mask;
+  a.row_loss = k.row_loss;
+  a.row_flags = k.row_flags;
+  a.hdr = k.hdr;
+  a.partials = k.partials;
+  a.rows_total = k.rows_total;
+  a.row_begin = k.row_begin;
+  a.row_end = k.row_end;
+  a.classes = k.classes;
+  a.row_stride = k.row_stride;
+  a.n = k.n_peers + 1;
+  a.pairwise = k.peer_reduce == CODISTILL_PEERS_PAIRWISE_MEAN;
+  a.reduction = k.reduction;
+  a.centred = k.dist == CODISTILL_DIST_MSE_CENTRED;
+  a.alpha = k.alpha;
+  a.eps = k.eps;
+  a.temperature = k.temperature;
+  int mode = kClMse;
+  if (k.dist == CODISTILL_DIST_KL_SOFTMAX)
+    mode = (k.peer_reduce == CODISTILL_PEERS_PAIRWISE_MEAN || k.n_peers == 1) ? kClKlPairwise : kClKlMeanTarget;
+  return launch_cluster(a, dtype, mode, false, smem_optin, stream);
+}
+
+}  // namespace codistill

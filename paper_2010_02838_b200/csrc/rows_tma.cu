@@ -23,6 +23,7 @@
 // is not a multiple of 16 start at varying offsets `head` inside their first segment.  Segments
 // that are only partly inside the row ("edge" segments) take a masked slow path.  Every valid row
 // uses the same number of pieces (some possibly empty), so that barrier phases advance uniformly.
+#include "bulk_copy.cuh"
 #include "common.cuh"
 #include "seg_math.cuh"
 
@@ -74,46 +75,6 @@ struct Ctrl {  // lives at the start of dynamic shared memory
   double fin[32];
 };
 static_assert(sizeof(Ctrl) <= kCtrlBytes - kZeroBytes, "control block fits its slot");
-
-// ------------------------------------------------------------------ PTX wrappers
-__device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
-__device__ __forceinline__ void mbar_init(uint64_t* bar, uint32_t count) {
-  asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(smem_u32(bar)), "r"(count) : "memory");
-}
-__device__ __forceinline__ void mbar_arrive(uint64_t* bar) {
-  asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_u32(bar)) : "memory");
-}
-__device__ __forceinline__ void mbar_arrive_expect_tx(uint64_t* bar, uint32_t bytes) {
-  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(smem_u32(bar)), "r"(bytes) : "memory");
-}
-__device__ __forceinline__ bool mbar_try_wait(uint64_t* bar, uint32_t parity) {
-  uint32_t ok;
-  asm volatile(
-      "{\n\t.reg .pred p;\n\t"
-      "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
-      "selp.u32 %0, 1, 0, p;\n\t}"
-      : "=r"(ok)
-      : "r"(smem_u32(bar)), "r"(parity)
-      : "memory");
-  return ok != 0;
-}
-// global -> shared bulk copy (no multicast); dst, src and bytes are multiples of 16
-__device__ __forceinline__ void bulk_g2s(void* dst, const void* src, uint32_t bytes, uint64_t* bar) {
-  asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];" ::"r"(
-                   smem_u32(dst)),
-               "l"(src), "r"(bytes), "r"(smem_u32(bar))
-               : "memory");
-}
-// shared -> global bulk copy; dst, src and bytes are multiples of 16.  Completion is tracked by the
-// issuing thread's bulk async-group.
-__device__ __forceinline__ void bulk_s2g(void* dst, const void* src, uint32_t bytes) {
-  asm volatile("cp.async.bulk.global.shared::cta.bulk_group [%0], [%1], %2;" ::"l"(dst), "r"(smem_u32(src)), "r"(bytes) : "memory");
-}
-__device__ __forceinline__ unsigned long long global_timer_ns() {
-  unsigned long long t;
-  asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
-  return t;
-}
 
 // Wait for a phase of an mbarrier, but never for ever: after kWaitLimitNs the CTA-wide abort flag
 // and the device status are set and every later wait returns at once (results are then invalid).
@@ -330,11 +291,11 @@ rows_tma_kernel(const __grid_constant__ KArgs a, const TmaCfg cfg) {
     for (int s = 0; s < 2; ++s) { mbar_init(&ctrl->end_full[s], NCW); mbar_init(&ctrl->end_empty[s], 1); }
     ctrl->abort_flag = 0;
     ctrl->last_flag = 0;
-    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    mbar_init_fence();
   }
   char* zero_region = reinterpret_cast<char*>(smem_raw) + (kCtrlBytes - kZeroBytes);
   for (int i = threadIdx.x * 16; i < kZeroBytes; i += blockDim.x * 16) *reinterpret_cast<uint4*>(zero_region + i) = make_uint4(0u, 0u, 0u, 0u);
-  asm volatile("fence.proxy.async.shared::cta;" ::: "memory");  // the zeros are read by bulk copies later
+  fence_proxy_async_shared();  // the zeros are read by bulk copies later
   wait_for_prior_grid();  // from here on the workspace header and the valid-row counts are read
   __syncthreads();
 
@@ -410,7 +371,7 @@ rows_tma_kernel(const __grid_constant__ KArgs a, const TmaCfg cfg) {
           if (lane == 0) {
             const uint32_t lo = (uint32_t)g.seg_lo * 16u, hi = (uint32_t)g.seg_hi * 16u;
             for (uint32_t o = lo; o < hi; o += kZeroBytes) bulk_s2g(g_img + o, zero_region, hi - o < (uint32_t)kZeroBytes ? hi - o : (uint32_t)kZeroBytes);
-            asm volatile("cp.async.bulk.commit_group;" ::: "memory");
+            bulk_commit_group();
           }
           if (lane < 2) {
             const int s = lane == 0 ? 0 : g.n_seg - 1;
@@ -444,7 +405,7 @@ rows_tma_kernel(const __grid_constant__ KArgs a, const TmaCfg cfg) {
     // results of the last two valid rows
     if (v >= 2) finish_row(v - 2, prev_row[v & 1]);
     if (v >= 1) finish_row(v - 1, prev_row[(v - 1) & 1]);
-    if (lane == 0) asm volatile("cp.async.bulk.wait_group 0;" ::: "memory");  // zero rows are written
+    if (lane == 0) bulk_wait_all_groups();  // zero rows are written
     // Before leaving, make sure no copy armed by this warp is still in flight (bounded).
     if (v >= 1)
       for (int k = 0; k < n_pieces; ++k) wait_bounded(&ctrl->own_full[k], (v - 1) & 1, ctrl, a.hdr);

@@ -37,10 +37,14 @@ def full_workload(idx):
 
 def check_gradient_rows(grad, ref_rows, mask, lo, n_valid):
     g = grad[lo:lo + 32].double().cpu().numpy()
-    # under the mean every element is scaled by 1/n_valid: compare at that scale (values whose
-    # scaled magnitude exceeds 1 are bounded by bf16 rounding itself, as in helpers.compare)
+    # under the mean every element is scaled by 1/n_valid: compare at that scale.  The stored value
+    # is the bf16 rounding of the element itself (about 1/n_valid in size), so the rounding step that
+    # bounds large elements is the step at the stored value, brought to the same scale.
     err = np.abs(g - ref_rows) * n_valid
-    assert np.all(err <= np.maximum(2e-3, 0.75 * bf16_ulp(ref_rows * n_valid))), float(err.max())
+    excess = err - np.maximum(2e-3, 0.75 * bf16_ulp(ref_rows) * n_valid)
+    worst = np.unravel_index(np.argmax(excess), excess.shape)
+    assert excess[worst] <= 0, (f"row {lo + worst[0]} column {worst[1]}: kernel {g[worst] * n_valid!r}, "
+                                f"oracle {ref_rows[worst] * n_valid!r} (both times n_valid)")
     dead = np.flatnonzero(mask[lo:lo + 32] == 0)
     assert np.all(g[dead] == 0)
 
