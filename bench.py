@@ -48,6 +48,10 @@ def parse_args():
     ap.add_argument("--e2e-steps", type=int, default=3)
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--sustain", type=float, default=3.0,
+                    help="seconds of back-to-back steps timed in chunks with the SM clock read after each (0: skip)")
+    ap.add_argument("--no-extras", action="store_true",
+                    help="skip the legs beside the headline (sustained run, graph replay, basic entry point)")
     return ap.parse_args()
 
 
@@ -130,18 +134,24 @@ def kernel_source_hash(files):
     return h.hexdigest()[:16]
 
 
-def stored_traffic(workload_idx, dist):
-    """DRAM bytes per launch from the committed ncu summary, or None when the kernel sources changed since."""
+def stored_traffic(workload_idx, dist, all_models, w):
+    """DRAM bytes per launch of the dominant kernel from the committed ncu record (profiles/dram_traffic.json),
+    or None when there is no record or the kernel sources changed since the capture.  A record holds the
+    counters of the second of two consecutive launches (caches left alone between them) on a reduced batch of
+    the same recipe; reads are scaled by valid rows, writes by rows."""
     path = os.path.join(ROOT, "profiles", "dram_traffic.json")
     if not os.path.exists(path):
         return None
     try:
-        rec = json.load(open(path)).get(f"config{workload_idx}_{dist}")
-        if rec and rec.get("source_hash") == kernel_source_hash(rec["sources"]):
-            return rec["dram_bytes_per_launch"]
+        rec = json.load(open(path)).get(f"config{workload_idx}_{dist}" + ("_all" if all_models else ""))
+        if not rec or rec.get("source_hash") != kernel_source_hash(rec["sources"]):
+            return None
+        cap = rec["capture"]
+        reads = cap["dram_bytes_read"] * (w.rows - w.n_padded) / cap["valid_rows"]
+        writes = cap["dram_bytes_write"] * w.rows / cap["rows"]
+        return int(reads + writes)
     except Exception:
-        pass
-    return None
+        return None
 
 
 # ------------------------------------------------------------------ reference arm: the CPU oracle
@@ -291,6 +301,10 @@ def run_ours(args):
     if status != 0:
         raise RuntimeError(f"device status {status} after the timed region")
 
+    extras = {}
+    if rank == 0 and world == 1 and not args.no_extras:
+        extras = run_extras(args, w, plan, models, labels, mask, cb, torch, stream, ms_step, local_rank)
+
     # ---- end to end through the host-buffer entry point (pinned host memory, copies inside the timed region)
     e2e = None
     if not args.no_e2e and not args.all_models:
@@ -322,12 +336,15 @@ def run_ours(args):
         "hbm_gbs_algorithmic": achieved,
         "hbm_gbs_dense_formula": None if args.all_models else w.algorithmic_bytes() / (ms_step * 1e-3) / 1e9,
         "roofline": {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
-                     "traffic": None if args.all_models else stored_traffic(args.workload, args.dist), "peak_source": peak_src,
+                     "traffic": stored_traffic(args.workload, args.dist, args.all_models, w), "peak_source": peak_src,
                      "bytes_per_launch": alg_bytes,
                      "note": note},
         "frac_of_nominal_8TBs": achieved / 8000.0,
         "clocks": clocks, "e2e": e2e, "gpu_launches": launches_per_step * args.steps,
     }
+    if clocks and clocks.get("sm_mhz"):
+        line["ms_x_sm_mhz"] = ms_step * clocks["sm_mhz"]     # for an issue-bound kernel: SM cycles per step / 1000
+    line.update(extras)
     if not args.no_cpu_baseline:
         v, dt, rows, cores, calls = time_oracle(w0, args.dist, 2, 1, min_seconds=12.0)
         line["cpu_baseline"] = {"value": v, "unit": UNIT, "cores": cores, "kind": "oracle",
@@ -336,6 +353,94 @@ def run_ours(args):
     print(json.dumps(line), flush=True)
     if world > 1:
         dist_pkg.destroy_process_group()
+
+
+def sm_clock_reader(index):
+    """Returns a function that reads the current SM clock in MHz through NVML (reading only), or None."""
+    try:
+        import pynvml
+        pynvml.nvmlInit()
+        handle = pynvml.nvmlDeviceGetHandleByIndex(index)
+        return lambda: int(pynvml.nvmlDeviceGetClockInfo(handle, pynvml.NVML_CLOCK_SM))
+    except Exception:
+        return None
+
+
+def run_extras(args, w, plan, models, labels, mask, cb, torch, stream, ms_step, device_index):
+    """Legs beside the headline, each timed with CUDA events on the launch stream:
+    - sustained: back-to-back steps for args.sustain seconds in chunks of about 50 ms, the SM clock read
+      after each chunk; time per step by clock bin, so that the dependence on the clock is on record;
+    - graph_replay (workloads that fit the L2, where launch latency dominates): the same call captured in a
+      CUDA graph, 20 steps per graph;
+    - basic_entry_point: the plain codistill_loss_fwd_bwd call (scratch from the stream-ordered allocator,
+      no counters) on the same tensors, single-model workloads with dense MSE only."""
+    out = {}
+    ev = lambda: torch.cuda.Event(enable_timing=True)
+    if args.sustain > 0:
+        read_clock = sm_clock_reader(device_index)
+        chunk = max(1, int(50.0 / max(ms_step, 1e-3)))
+        bins, t_all, t0 = {}, [], time.perf_counter()
+        while time.perf_counter() - t0 < args.sustain:
+            e0, e1 = ev(), ev()
+            e0.record(stream)
+            for _ in range(chunk):
+                plan.run(stream)
+            e1.record(stream)
+            e1.synchronize()
+            mhz = read_clock() if read_clock else None
+            ms = e0.elapsed_time(e1) / chunk
+            t_all.append(ms)
+            bins.setdefault(mhz, []).append(ms)
+        t_all.sort()
+        out["sustained"] = {
+            "seconds": round(time.perf_counter() - t0, 2), "steps": chunk * len(t_all),
+            "ms_per_step_median": t_all[len(t_all) // 2], "ms_per_step_max": t_all[-1],
+            "by_sm_mhz": {str(k): {"chunks": len(v), "ms_per_step_median": sorted(v)[len(v) // 2]}
+                          for k, v in sorted(bins.items(), key=lambda kv: -(kv[0] or 0))},
+            "note": "chunks of about 50 ms of back-to-back steps; SM clock read through NVML after each chunk"}
+    if w.algorithmic_bytes() <= 3 * 126e6:
+        try:
+            per_graph = 20
+            side = torch.cuda.Stream()
+            side.wait_stream(stream)
+            with torch.cuda.stream(side):
+                plan.run(side)
+            stream.wait_stream(side)
+            torch.cuda.synchronize()
+            g = torch.cuda.CUDAGraph()
+            with torch.cuda.graph(g):
+                for _ in range(per_graph):
+                    plan.run(torch.cuda.current_stream())
+            for _ in range(3):
+                g.replay()
+            reps = max(5, args.steps // per_graph)
+            e0, e1 = ev(), ev()
+            e0.record()
+            for _ in range(reps):
+                g.replay()
+            e1.record()
+            e1.synchronize()
+            out["graph_replay"] = {"ms_per_step": e0.elapsed_time(e1) / (reps * per_graph), "steps_per_graph": per_graph,
+                                   "replays": reps, "note": "the same C-ABI call captured in a CUDA graph"}
+        except Exception as exc:   # capture is a convenience of this benchmark, not of the library's contract
+            out["graph_replay"] = {"error": str(exc)[:200]}
+    if not args.all_models and args.dist == "mse":
+        outs = cb.Outputs(torch.empty(w.rows, dtype=torch.float32, device="cuda"),
+                          torch.empty(1, dtype=torch.float32, device="cuda"), torch.empty_like(models[0]), None, None)
+        call = lambda: cb.codistill_loss_fwd_bwd(models[0], models[1:], labels, mask, alpha=w.alpha,
+                                                 temperature=w.temperature, out=outs, stream=stream)
+        for _ in range(3):
+            call()
+        e0, e1 = ev(), ev()
+        e0.record(stream)
+        for _ in range(args.steps):
+            call()
+        e1.record(stream)
+        e1.synchronize()
+        out["basic_entry_point"] = {"ms_per_step": e0.elapsed_time(e1) / args.steps, "api": "codistill_loss_fwd_bwd",
+                                    "note": "same tensors; this call has no label smoothing and no counters, and takes "
+                                            "its scratch from the stream-ordered allocator"}
+    return out
 
 
 def run_e2e(args, w, models, labels, mask, cb, torch, world, barrier, dist_code):
@@ -385,10 +490,24 @@ def run_e2e(args, w, models, labels, mask, cb, torch, world, barrier, dist_code)
             "api": "codistill_loss_fwd_bwd_host (pinned host buffers, copies inside the timed region)"}
 
 
+def torchrun_command(argv, gpus, port=None):
+    """The command that runs this script as one process per GPU of this node."""
+    if port is None:
+        import socket
+        with socket.socket() as s:
+            s.bind(("127.0.0.1", 0))
+            port = s.getsockname()[1]
+    return [sys.executable, "-m", "torch.distributed.run", "--nnodes=1", f"--nproc-per-node={gpus}",
+            "--master-addr", "127.0.0.1", "--master-port", str(port), os.path.abspath(__file__), *argv]
+
+
 def main():
     args = parse_args()
     if args.impl == "reference":
         run_reference(args)
+    elif args.gpus > 1 and "WORLD_SIZE" not in os.environ:
+        # asked for N GPUs outside a launcher: start one rank per GPU and let rank 0 print the line
+        os.execvp(sys.executable, torchrun_command(sys.argv[1:], args.gpus))
     else:
         run_ours(args)
 

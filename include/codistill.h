@@ -8,8 +8,8 @@
  *
  *     loss_row = L(y, z) + alpha * 1/(n-1) * sum_{j != i} D(z, z^(j))
  *
- * where L is the cross-entropy of softmax(z) against the label y (Section 2: "a standard
- * supervised loss function L (e.g., cross-entropy ...)") and D is, as in the paper's
+ * where L is the supervised loss of Section 2, here the cross-entropy of softmax(z) against the
+ * label y (the paper's experiments are all classification), and D is, as in the paper's
  * experiments (Appendix, "Implementation Details"), the mean squared error between the raw,
  * un-centred logits of the two models.  The KL divergence between temperature softmaxes
  * that Section 2 attributes to earlier work is available as a second form of D.  The
@@ -210,8 +210,8 @@ size_t codistill_workspace_bytes(int n, int64_t rows, int64_t classes, int dtype
 size_t codistill_host_workspace_bytes(int n, int64_t rows, int64_t classes, int dtype, int64_t chunk_rows);
 
 /*
- * All models in one call: Algorithm 1 updates every model i = 1..n on the same minibatch ("for i = 1,
- * ..., n in parallel"), and each update needs the objective with model i as "own" and the other n-1 as
+ * All models in one call: Algorithm 1 updates every model i = 1..n on the same minibatch (its inner
+ * loop over the models), and each update needs the objective with model i as "own" and the other n-1 as
  * peers.  Done with n calls above, every logit tensor is read n times and n gradients are written:
  * n (n + 1) tensor passes.  This entry point computes the n objectives together: the per-column sums
  * over the models are shared, so that 3 n passes suffice (each tensor read twice, each gradient
@@ -264,6 +264,23 @@ size_t codistill_all_workspace_bytes(int n, int64_t rows);
 /* Human-readable name of a CODISTILL_ERR_* code (static storage). */
 const char* codistill_status_string(int status);
 
+/*
+ * Diagnostic, not part of the objective.  Every wait of the kernels on an asynchronous copy is bounded:
+ * when its time limit runs out the kernel raises CODISTILL_DEV_TIMEOUT in the status word, stops waiting
+ * and leaves normally; the context stays usable.  This call shows that path without a copy that never
+ * lands: it launches one small CTA that waits `limit_ns` nanoseconds (1 .. 100 000 000) on a barrier
+ * that nothing completes, then writes the status bits to *dev_status (DEVICE pointer; expected value
+ * CODISTILL_DEV_TIMEOUT).  Asynchronous on `stream` like every call.
+ */
+int codistill_selftest_bounded_wait(int32_t* dev_status, uint64_t limit_ns, void* stream);
+
+/*
+ * Text of the CUDA runtime error behind the most recent CODISTILL_ERR_CUDA on this host thread
+ * ("no error" when there was none).  The library carries its own copy of the CUDA runtime, so the
+ * error is not visible through the caller's cudaGetLastError.  Reading it clears it.  Static storage.
+ */
+const char* codistill_last_cuda_error(void);
+
 /* Library version: major * 10000 + minor * 100 + patch. */
 int codistill_version(void);
 
@@ -271,10 +288,13 @@ int codistill_version(void);
  * Name of the kernel regime the dispatcher picks for a problem, so that tests and benchmarks can
  * state which kernel they exercised: "warp" (rows up to 8 KiB, one warp per row), "tma" (long rows,
  * MSE distance, own row staged in shared memory by bulk copies), "stream" (long rows, direct loads,
- * own row read twice; MSE rows beyond 64 KiB and the KL distance) or "block" (everything else).  The
- * answer assumes 16-byte aligned tensor bases (the long-row kernels need them).  The environment
- * variable CODISTILL_REGIME = tma | stream | block overrides the choice where the named kernel can
- * serve the call.  Static storage; NULL on bad arguments.
+ * own row read twice: MSE rows beyond 64 KiB, calls without peers), "cluster" (long rows, all n row
+ * images of a row index kept in the shared memory of a thread-block cluster: the softmax-KL and
+ * centred-MSE distances, and MSE with 4 to 6 peers) or "block" (everything else).  The answer assumes
+ * 16-byte aligned tensor bases (the long-row kernels need them).  For measurements the environment
+ * variable CODISTILL_REGIME = tma | stream | cluster | block overrides the choice where the named
+ * kernel can serve the call, and CODISTILL_CLUSTER_SIZE = 1 | 2 | 4 | 8 | 16 fixes the number of
+ * CTAs per cluster of the "cluster" kernel.  Static storage; NULL on bad arguments.
  */
 const char* codistill_kernel_regime(int n, int64_t rows, int64_t classes, int64_t row_stride, int dtype,
                                     int dist_kind, int peer_reduce);

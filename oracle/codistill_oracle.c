@@ -18,8 +18,11 @@
  *     squared error, i.e. the variance over the classes of the difference) is dist_kind 2.
  *   - Section 3 / Section 5: the term may be omitted (non-communication steps), n = 1 is
  *     ordinary training.
- * Readings where the paper is silent (label smoothing target, padding mask, temperature and
- * the T^2 factor of the KL form, reduction over rows, arg-max ties) are listed in the design doc.
+ * Readings where the paper is silent: label smoothing is uniform, q = (1 - eps) onehot(y) + eps / C;
+ * a padding mask is one byte per row (non-zero = valid), masked rows give zero loss and gradient;
+ * the KL form is T^2 KL(softmax(peer / T) || softmax(own / T)) with the peer as target; the reduced
+ * loss is the mean over valid rows (or the sum) and the gradient is the gradient of that; the first
+ * (lowest) index wins arg-max ties and -0.0 ties with +0.0.
  *
  * Pins: every function here is pinned by tests/test_oracle_pins.py (closed forms, a hand
  * example, invariants, finite differences, a float64 autograd composition of library ops,

@@ -23,13 +23,18 @@ REDUCE_MEAN_VALID, REDUCE_SUM = 0, 1
 DEV_BAD_LABEL, DEV_TIMEOUT, DEV_ASSERT = 1, 2, 4
 MAX_PEERS = 31
 STATIC_MAX_ROWS = 65536
+ERR_CUDA = 6
 ERR_TOO_LARGE = 8
 
 EXPORTS = (
     "codistill_loss_fwd_bwd", "codistill_loss_fwd_bwd_ex", "codistill_loss_fwd_bwd_host",
     "codistill_loss_fwd_bwd_static", "codistill_loss_fwd_bwd_all", "codistill_all_workspace_bytes",
     "codistill_workspace_bytes", "codistill_host_workspace_bytes", "codistill_status_string",
-    "codistill_version", "codistill_kernel_regime",
+    "codistill_version", "codistill_kernel_regime", "codistill_last_cuda_error",
+    "codistill_selftest_bounded_wait",
+    "codistill_schedule_alpha", "codistill_schedule_piecewise", "codistill_schedule_step_decay",
+    "codistill_is_exchange_step", "codistill_bits_all_reduce", "codistill_bits_checkpoints",
+    "codistill_bits_predictions",
 )
 
 
@@ -93,7 +98,8 @@ class AllParams(ctypes.Structure):
 class CodistillError(RuntimeError):
     def __init__(self, code: int):
         self.code = code
-        super().__init__(f"codistill error {code}: {status_string(code)}")
+        detail = f" ({load_library().codistill_last_cuda_error().decode()})" if code == ERR_CUDA else ""
+        super().__init__(f"codistill error {code}: {status_string(code)}{detail}")
 
 
 _lib = None
@@ -128,10 +134,29 @@ def load_library() -> ctypes.CDLL:
     lib.codistill_host_workspace_bytes.argtypes = [i32, i64, i64, i32, i64]
     lib.codistill_status_string.restype = ctypes.c_char_p
     lib.codistill_status_string.argtypes = [i32]
+    lib.codistill_selftest_bounded_wait.restype = i32
+    lib.codistill_selftest_bounded_wait.argtypes = [vp, ctypes.c_uint64, vp]
+    lib.codistill_last_cuda_error.restype = ctypes.c_char_p
+    lib.codistill_last_cuda_error.argtypes = []
     lib.codistill_version.restype = i32
     lib.codistill_version.argtypes = []
     lib.codistill_kernel_regime.restype = ctypes.c_char_p
     lib.codistill_kernel_regime.argtypes = [i32, i64, i64, i64, i32, i32, i32]
+    f64, pd, pi64 = ctypes.c_double, ctypes.POINTER(ctypes.c_double), ctypes.POINTER(ctypes.c_int64)
+    lib.codistill_schedule_alpha.restype = f64
+    lib.codistill_schedule_alpha.argtypes = [f64, f64, i64]
+    lib.codistill_schedule_piecewise.restype = f64
+    lib.codistill_schedule_piecewise.argtypes = [pd, pi64, i32, i64]
+    lib.codistill_schedule_step_decay.restype = f64
+    lib.codistill_schedule_step_decay.argtypes = [f64, f64, pi64, i32, i64]
+    lib.codistill_is_exchange_step.restype = i32
+    lib.codistill_is_exchange_step.argtypes = [i64, i64]
+    lib.codistill_bits_all_reduce.restype = f64
+    lib.codistill_bits_all_reduce.argtypes = [f64]
+    lib.codistill_bits_checkpoints.restype = f64
+    lib.codistill_bits_checkpoints.argtypes = [i32, f64, i64]
+    lib.codistill_bits_predictions.restype = f64
+    lib.codistill_bits_predictions.argtypes = [i32, i64, i32, i64, i64]
     _lib = lib
     return lib
 
@@ -375,3 +400,52 @@ class AllPlan:
         if rc != OK:
             raise CodistillError(rc)
         return self.out
+
+
+def selftest_bounded_wait(limit_ns: int = 1_000_000, stream: torch.cuda.Stream | None = None) -> torch.Tensor:
+    """Diagnostic: one CTA waits `limit_ns` on a barrier nothing completes; returns the [1] int32 status tensor."""
+    status = torch.zeros(1, dtype=torch.int32, device="cuda")
+    rc = load_library().codistill_selftest_bounded_wait(_ptr(status), int(limit_ns), _stream_ptr(stream))
+    if rc != OK:
+        raise CodistillError(rc)
+    return status
+
+
+# ------------------------------------------------------------------ host-side schedules (codistill_schedule.h)
+def schedule_alpha(alpha0: float, gamma: float, epoch: int) -> float:
+    return float(load_library().codistill_schedule_alpha(float(alpha0), float(gamma), int(epoch)))
+
+
+def _i64_array(xs):
+    xs = [int(x) for x in xs]
+    return (ctypes.c_int64 * max(1, len(xs)))(*xs), len(xs)
+
+
+def schedule_piecewise(values, milestones, epoch: int) -> float:
+    vals = (ctypes.c_double * len(values))(*[float(v) for v in values])
+    ms, n = _i64_array(milestones)
+    if len(values) != n + 1:
+        raise ValueError("values must have one entry more than milestones")
+    return float(load_library().codistill_schedule_piecewise(vals, ms, n, int(epoch)))
+
+
+def schedule_step_decay(base: float, factor: float, milestones, epoch: int) -> float:
+    ms, n = _i64_array(milestones)
+    return float(load_library().codistill_schedule_step_decay(float(base), float(factor), ms, n, int(epoch)))
+
+
+def is_exchange_step(step: int, period: int) -> bool:
+    return bool(load_library().codistill_is_exchange_step(int(step), int(period)))
+
+
+def bits_all_reduce(b_model: float) -> float:
+    return float(load_library().codistill_bits_all_reduce(float(b_model)))
+
+
+def bits_checkpoints(n: int, b_model: float, period: int) -> float:
+    return float(load_library().codistill_bits_checkpoints(int(n), float(b_model), int(period)))
+
+
+def bits_predictions(n: int, classes: int, bits_per_value: int, batch_per_device: int, period: int) -> float:
+    return float(load_library().codistill_bits_predictions(int(n), int(classes), int(bits_per_value),
+                                                           int(batch_per_device), int(period)))

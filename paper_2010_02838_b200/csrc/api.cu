@@ -1,12 +1,14 @@
 // Host side of the C ABI declared in include/codistill.h: argument validation, workspace
 // layout, regime dispatch, the prep / finalize kernels and the host-buffer pipeline.
 #include <math.h>
+#include <stdio.h>
 #include <stdlib.h>
 #include <string.h>
 
 #include <atomic>
 #include <mutex>
 
+#include "bulk_copy.cuh"
 #include "common.cuh"
 
 static_assert(sizeof(codistill_params_t) == 152, "ABI: size of codistill_params_t");
@@ -21,6 +23,20 @@ bool stream_supported(const KArgs& a, int dtype);
 cudaError_t launch_stream(const KArgs& a, int dtype, int num_sms, cudaStream_t stream);
 bool cluster_supported(const KArgs& a, int dtype, int smem_optin);
 cudaError_t launch_cluster_single(const KArgs& a, int dtype, int smem_optin, cudaStream_t stream);
+
+static thread_local cudaError_t g_last_cuda_error = cudaSuccess;
+static thread_local const char* g_last_cuda_call = "";
+static thread_local char g_last_cuda_text[256];
+cudaError_t cuda_note(cudaError_t e, const char* what) {
+  if (e != cudaSuccess) g_last_cuda_call = what;
+  return e;
+}
+int cuda_status(cudaError_t e) {
+  if (e == cudaSuccess) return CODISTILL_OK;
+  g_last_cuda_error = e;
+  cudaGetLastError();   // a launch failure also sits in the runtime's own slot: clear it
+  return CODISTILL_ERR_CUDA;
+}
 
 // ------------------------------------------------------------------ prep and finalize kernels
 // Zeroes the workspace header and counts valid / masked rows (one partial pair per block, summed
@@ -74,6 +90,23 @@ static_assert(kPrepMaxBlocks <= 59, "per-block bad-label words live in the heade
 __global__ void __launch_bounds__(1024) finalize_kernel(const __grid_constant__ KArgs a) {
   __shared__ double sh[32];
   finalize_cta(a, sh);
+}
+
+// Diagnostic: one CTA waits, with the library's bounded wait, on an mbarrier that nothing ever completes
+// (no copy is in flight, so the CTA may leave at once afterwards).  Shows that an expired wait ends in a
+// status bit and a normal kernel exit.
+__global__ void __launch_bounds__(64) bounded_wait_probe_kernel(int32_t* dev_status, unsigned long long limit_ns) {
+  __shared__ uint64_t bar;
+  __shared__ int abort_flag;
+  if (threadIdx.x == 0) {
+    mbar_init(&bar, 1);
+    mbar_init_fence();
+    abort_flag = 0;
+    *dev_status = 0;
+  }
+  __syncthreads();
+  // warp 0 polls back to back like a consumer, warp 1 with back-off like a producer
+  mbar_wait_limited(&bar, 0u, &abort_flag, dev_status, CODISTILL_DEV_TIMEOUT, limit_ns, true, threadIdx.x >= 32);
 }
 
 // ------------------------------------------------------------------ host helpers
@@ -145,6 +178,7 @@ static Regime pick_regime(const KArgs& a, int dtype, int smem_optin) {
   if (can_cluster && a.dist != CODISTILL_DIST_MSE_LOGITS) return kRegimeCluster;
   if (can_tma && (!can_stream || tma_ctas_per_sm(a, dtype, smem_optin) >= 2)) return kRegimeTma;
   if (can_stream) return kRegimeStream;
+  if (can_cluster) return kRegimeCluster;   // peer counts the two MSE kernels above are not built for (4, 5, 6)
   return generic;
 }
 
@@ -224,16 +258,16 @@ static cudaError_t launch_main(const KArgs& a, int dtype, const DeviceInfo& di, 
 static int run_device(const codistill_params_t* p, cudaStream_t stream) {
   if (p->workspace_bytes < ws_layout(p->rows).total) return CODISTILL_ERR_WORKSPACE;
   DeviceInfo di;
-  if (device_info(&di) != cudaSuccess) return CODISTILL_ERR_CUDA;
+  if (const int rc_cuda = cuda_status(device_info(&di))) return rc_cuda;
   KArgs a;
   fill_args(&a, p, p->workspace);
-  if (launch_prep(a, stream) != cudaSuccess) return CODISTILL_ERR_CUDA;
+  if (const int rc_cuda = cuda_status(launch_prep(a, stream))) return rc_cuda;
   if (p->rows == 0) {
     a.fused_finalize = 0;
     finalize_kernel<<<1, 1024, 0, stream>>>(a);
-    return cudaGetLastError() == cudaSuccess ? CODISTILL_OK : CODISTILL_ERR_CUDA;
+    return cuda_status(cudaGetLastError());
   }
-  if (launch_main(a, p->dtype, di, stream) != cudaSuccess) return CODISTILL_ERR_CUDA;
+  if (const int rc_cuda = cuda_status(launch_main(a, p->dtype, di, stream))) return rc_cuda;
   return CODISTILL_OK;
 }
 
@@ -270,14 +304,14 @@ static HostLayout host_layout(int n, int64_t rows, int64_t row_stride, int dtype
   return h;
 }
 
-#define CODISTILL_CK(expr) do { if ((expr) != cudaSuccess) { rc = CODISTILL_ERR_CUDA; goto done; } } while (0)
+#define CODISTILL_CK(expr) do { if ((rc = cuda_status(expr)) != CODISTILL_OK) goto done; } while (0)
 
 static int run_host(const codistill_params_t* p, int64_t chunk_rows_req, cudaStream_t stream) {
   const size_t es = p->dtype == CODISTILL_F32 ? 4 : 2;
   const HostLayout h = host_layout(p->n, p->rows, p->row_stride, p->dtype, chunk_rows_req);
   if (p->workspace_bytes < h.total) return CODISTILL_ERR_WORKSPACE;
   DeviceInfo di;
-  if (device_info(&di) != cudaSuccess) return CODISTILL_ERR_CUDA;
+  if (const int rc_cuda = cuda_status(device_info(&di))) return rc_cuda;
   char* base = static_cast<char*>(p->workspace);
   const int64_t R = p->rows;
   const int P = p->n - 1;
@@ -373,7 +407,22 @@ using namespace codistill;
 
 extern "C" {
 
-int codistill_version(void) { return 100; }
+int codistill_version(void) { return 200; }
+
+int codistill_selftest_bounded_wait(int32_t* dev_status, uint64_t limit_ns, void* stream) {
+  if (dev_status == nullptr) return CODISTILL_ERR_NULL;
+  if (limit_ns == 0 || limit_ns > 100000000ull) return CODISTILL_ERR_PARAM;   // at most 100 ms
+  bounded_wait_probe_kernel<<<1, 64, 0, static_cast<cudaStream_t>(stream)>>>(dev_status, limit_ns);
+  return cuda_status(cudaGetLastError());
+}
+
+const char* codistill_last_cuda_error(void) {
+  const cudaError_t e = g_last_cuda_error;
+  snprintf(g_last_cuda_text, sizeof(g_last_cuda_text), "%s%s%s", cudaGetErrorString(e), g_last_cuda_call[0] ? " in " : "", g_last_cuda_call);
+  g_last_cuda_error = cudaSuccess;
+  g_last_cuda_call = "";
+  return g_last_cuda_text;
+}
 
 const char* codistill_status_string(int status) {
   switch (status) {
@@ -433,11 +482,11 @@ int codistill_loss_fwd_bwd(const void* logits, const void* const* peer_logits, c
   cudaStream_t s = static_cast<cudaStream_t>(stream);
   const size_t bytes = ws_layout(rows).total;
   void* ws = nullptr;
-  if (cudaMallocAsync(&ws, bytes, s) != cudaSuccess) return CODISTILL_ERR_CUDA;
+  if (const int rc_cuda = cuda_status(cudaMallocAsync(&ws, bytes, s))) return rc_cuda;
   p.workspace = ws;
   p.workspace_bytes = bytes;
   const int rc = run_device(&p, s);
-  if (cudaFreeAsync(ws, s) != cudaSuccess) return CODISTILL_ERR_CUDA;
+  if (const int rc_cuda = cuda_status(cudaFreeAsync(ws, s))) return rc_cuda;
   return rc;
 }
 
@@ -494,14 +543,15 @@ static int static_scratch_address(void** out) {
   static std::atomic<void*> cache[64];
   static std::mutex fill;
   int dev = 0;
-  if (cudaGetDevice(&dev) != cudaSuccess) return CODISTILL_ERR_CUDA;
+  if (const int rc_cuda = cuda_status(cudaGetDevice(&dev))) return rc_cuda;
   const bool cached = dev >= 0 && dev < 64;
   if (cached) {
     if (void* known = cache[dev].load(std::memory_order_acquire)) { *out = known; return CODISTILL_OK; }
   }
   std::lock_guard<std::mutex> lock(fill);
   void* ptr = nullptr;
-  if (cudaGetSymbolAddress(&ptr, g_static_scratch) != cudaSuccess || ptr == nullptr) return CODISTILL_ERR_CUDA;
+  if (const int rc_cuda = cuda_status(cudaGetSymbolAddress(&ptr, g_static_scratch))) return rc_cuda;
+  if (ptr == nullptr) return CODISTILL_ERR_CUDA;
   if (cached) cache[dev].store(ptr, std::memory_order_release);
   *out = ptr;
   return CODISTILL_OK;

@@ -51,4 +51,30 @@ __device__ __forceinline__ unsigned long long global_timer_ns() {
   return t;
 }
 
+// Bounded wait for a phase of an mbarrier.  Polls until the phase completes, or the CTA-wide abort flag is
+// up (only when heed_abort), or `limit_ns` nanoseconds of polling have gone by; in the last case it raises the
+// abort flag and ORs `timeout_bit` into *status.  Returns true when the phase completed.  With back_off the
+// thread sleeps between polls (for warps that have slack and should not take issue slots from others).
+// Kept out of line: callers try the barrier once inline and come here only when they really have to wait.
+static __device__ __noinline__ bool mbar_wait_limited(uint64_t* bar, uint32_t parity, volatile int* abort_flag, int* status,
+                                               int timeout_bit, unsigned long long limit_ns, bool heed_abort, bool back_off) {
+  uint32_t polls = 0;
+  unsigned long long t0 = 0;
+  while (!mbar_try_wait(bar, parity)) {
+    if (back_off) __nanosleep(128);
+    if ((++polls & 0x3FFu) == 0 || (back_off && (polls & 0x3Fu) == 0)) {
+      if (heed_abort && *abort_flag) return false;
+      const unsigned long long now = global_timer_ns();
+      if (t0 == 0) {
+        t0 = now;
+      } else if (now - t0 > limit_ns) {
+        *abort_flag = 1;
+        atomicOr(status, timeout_bit);
+        return false;
+      }
+    }
+  }
+  return true;
+}
+
 }  // namespace codistill

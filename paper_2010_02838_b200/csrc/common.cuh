@@ -69,6 +69,13 @@ struct KArgs {
   float alpha, temperature, eps;
 };
 
+// ------------------------------------------------------------------ CUDA errors
+// CODISTILL_OK for cudaSuccess; otherwise the error is kept for codistill_last_cuda_error() (per host
+// thread) and CODISTILL_ERR_CUDA is returned.  Defined in api.cu.
+int cuda_status(cudaError_t e);
+// Same, for code that hands a cudaError_t on: remembers which call failed (a string literal) and returns e.
+cudaError_t cuda_note(cudaError_t e, const char* what);
+
 // ------------------------------------------------------------------ programmatic dependent launch
 // The main kernels are launched with programmatic stream serialisation: their CTAs may start while
 // the prep kernel of the same call still runs, so that launch latency and set-up overlap with it.

@@ -1,4 +1,4 @@
-// All n models in one call (Algorithm 1's loop "for i = 1..n in parallel" over one minibatch):
+// All n models in one call (Algorithm 1's inner loop over the models i = 1..n, on one minibatch):
 // every model's objective with the other n-1 models as its peers, MSE-on-logits distance.
 //
 // (With the centred distance every model's logits first lose their mean over the classes, known after pass A.)
@@ -641,9 +641,9 @@ extern "C" int codistill_loss_fwd_bwd_all(const codistill_all_params_t* p, void*
   if (p->workspace_bytes < l.total) return CODISTILL_ERR_WORKSPACE;
 
   int dev = 0, num_sms = 0, smem_optin = 0;
-  if (cudaGetDevice(&dev) != cudaSuccess) return CODISTILL_ERR_CUDA;
-  if (cudaDeviceGetAttribute(&num_sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) return CODISTILL_ERR_CUDA;
-  if (cudaDeviceGetAttribute(&smem_optin, cudaDevAttrMaxSharedMemoryPerBlockOptin, dev) != cudaSuccess) return CODISTILL_ERR_CUDA;
+  if (const int rc_cuda = cuda_status(cudaGetDevice(&dev))) return rc_cuda;
+  if (const int rc_cuda = cuda_status(cudaDeviceGetAttribute(&num_sms, cudaDevAttrMultiProcessorCount, dev))) return rc_cuda;
+  if (const int rc_cuda = cuda_status(cudaDeviceGetAttribute(&smem_optin, cudaDevAttrMaxSharedMemoryPerBlockOptin, dev))) return rc_cuda;
 
   char* ws = static_cast<char*>(p->workspace);
   AllArgs a;
@@ -669,8 +669,7 @@ extern "C" int codistill_loss_fwd_bwd_all(const codistill_all_params_t* p, void*
   a.eps = p->label_smoothing;
   a.temperature = p->dist_kind == CODISTILL_DIST_KL_SOFTMAX ? p->temperature : 0.f;  // 0: one of the MSE forms
 
-  if (launch_prep_rows(a.hdr, const_cast<int64_t*>(a.partials), a.labels, a.mask, a.rows, a.classes, stream) != cudaSuccess)
-    return CODISTILL_ERR_CUDA;
+  if (const int rc_cuda = cuda_status(launch_prep_rows(a.hdr, const_cast<int64_t*>(a.partials), a.labels, a.mask, a.rows, a.classes, stream))) return rc_cuda;
   if (a.rows > 0) {
     // Long rows: the cluster-resident kernel reads every logit from HBM once (the n row images of a row
     // index stay in the shared memory of a cluster); the direct-load kernel above reads them twice.
@@ -704,8 +703,8 @@ extern "C" int codistill_loss_fwd_bwd_all(const codistill_all_params_t* p, void*
     } else {
       e = p->dtype == CODISTILL_F32 ? all_launch<float>(a, num_sms, stream) : all_launch<__nv_bfloat16>(a, num_sms, stream);
     }
-    if (e != cudaSuccess) return CODISTILL_ERR_CUDA;
+    if (const int rc_cuda = cuda_status(e)) return rc_cuda;
   }
   finalize_all_kernel<<<a.n, 1024, 0, stream>>>(a);
-  return cudaGetLastError() == cudaSuccess ? CODISTILL_OK : CODISTILL_ERR_CUDA;
+  return cuda_status(cudaGetLastError());
 }

@@ -49,6 +49,7 @@ constexpr int kClMaxCluster = 16;
 constexpr int kClCtrlBytes = 4096;
 constexpr uint32_t kClCopyPiece = 32768;
 constexpr unsigned long long kClWaitLimitNs = 2000000000ull;   // bounded waits: 2 s, then CODISTILL_DEV_TIMEOUT
+constexpr unsigned long long kClDrainLimitNs = 50000000ull;    // last wait of an aborted CTA: 50 ms
 
 // what one warp found in a sub-range of one tensor
 struct ClRec { float m; int seg; float S, sum_z, S_T; int tensor; };
@@ -75,27 +76,9 @@ static_assert(sizeof(ClCtrl) <= kClCtrlBytes, "control block fits its slot");
 
 // Wait for a phase of the copy barrier, but never for ever: after the limit the CTA-wide abort flag and the
 // device status are set and later waits return early (results are then invalid, control flow stays uniform).
-__device__ __noinline__ void cl_wait_slow(uint64_t* bar, uint32_t parity, ClCtrl* ctrl, WsHeader* hdr, bool heed_abort) {
-  volatile int* abort_flag = &ctrl->abort_flag;
-  uint32_t polls = 0;
-  unsigned long long t0 = 0;
-  while (!mbar_try_wait(bar, parity)) {
-    if ((++polls & 0x3FFu) == 0) {
-      if (heed_abort && *abort_flag) return;
-      const unsigned long long now = global_timer_ns();
-      if (t0 == 0) {
-        t0 = now;
-      } else if (now - t0 > kClWaitLimitNs) {
-        *abort_flag = 1;
-        atomicOr(&hdr->status, CODISTILL_DEV_TIMEOUT);
-        return;
-      }
-    }
-  }
-}
 __device__ __forceinline__ void cl_wait(uint64_t* bar, uint32_t parity, ClCtrl* ctrl, WsHeader* hdr) {
   if (mbar_try_wait(bar, parity)) return;
-  cl_wait_slow(bar, parity, ctrl, hdr, true);
+  mbar_wait_limited(bar, parity, &ctrl->abort_flag, &hdr->status, CODISTILL_DEV_TIMEOUT, kClWaitLimitNs, true, false);
 }
 
 // exp((z - m) / T) for a pair of columns; l2eT = log2(e) / T
@@ -673,7 +656,7 @@ __global__ void __launch_bounds__(kClThreads, 2) rows_cluster_kernel(const __gri
   if (rank == 0 && v >= 1) finish_row((v - 1) & 1);
   if (ctrl->abort_flag && tid == 0) {
     // a wait ran out: give copies that may still be in flight one more bounded interval before the CTA ends
-    cl_wait_slow(&ctrl->full, (uint32_t)(v + 1) & 1u, ctrl, a.hdr, false);
+    mbar_wait_limited(&ctrl->full, (uint32_t)(v + 1) & 1u, &ctrl->abort_flag, &a.hdr->status, CODISTILL_DEV_TIMEOUT, kClDrainLimitNs, false, true);
   }
   cluster.sync();
 }
@@ -721,11 +704,13 @@ ClPlan cluster_plan(int n, int64_t classes, int64_t row_stride, int dtype, int s
 template <typename T, int N, int MODE, bool ALL>
 static cudaError_t cluster_launch_one(const ClArgs& a, const ClPlan& p, cudaStream_t stream) {
   auto kernel = rows_cluster_kernel<T, N, MODE, ALL>;
-  // per kernel and launch shape: attributes set and the number of co-resident clusters asked once per device
+  // per kernel: the number of co-resident clusters of a launch shape is asked once per device, and the
+  // kernel's shared-memory limit is only ever raised (a lower value would refuse earlier, larger shapes)
   static std::mutex mu;
   static std::map<std::tuple<int, int, uint32_t>, int> known;
+  static std::map<int, uint32_t> smem_limit;
   int dev = 0;
-  cudaError_t e = cudaGetDevice(&dev);
+  cudaError_t e = cuda_note(cudaGetDevice(&dev), "cudaGetDevice");
   if (e != cudaSuccess) return e;
   cudaLaunchConfig_t cfg = {};
   cfg.blockDim = dim3(kClThreads);
@@ -748,11 +733,15 @@ static cudaError_t cluster_launch_one(const ClArgs& a, const ClPlan& p, cudaStre
     if (it != known.end()) {
       max_clusters = it->second;
     } else {
-      if ((e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)p.smem_bytes)) != cudaSuccess) return e;
-      if (p.cluster > 8 && (e = cudaFuncSetAttribute(kernel, cudaFuncAttributeNonPortableClusterSizeAllowed, 1)) != cudaSuccess) return e;
+      if (p.smem_bytes > smem_limit[dev]) {
+        if ((e = cuda_note(cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)p.smem_bytes),
+                           "cudaFuncSetAttribute (shared memory size, cluster kernel)")) != cudaSuccess) return e;
+        smem_limit[dev] = p.smem_bytes;
+      }
+      if (p.cluster > 8 && (e = cuda_note(cudaFuncSetAttribute(kernel, cudaFuncAttributeNonPortableClusterSizeAllowed, 1), "cudaFuncSetAttribute (cluster size)")) != cudaSuccess) return e;
       cfg.gridDim = dim3((unsigned)p.cluster);
-      if ((e = cudaOccupancyMaxActiveClusters(&max_clusters, kernel, &cfg)) != cudaSuccess) return e;
-      if (max_clusters < 1) return cudaErrorLaunchOutOfResources;
+      if ((e = cuda_note(cudaOccupancyMaxActiveClusters(&max_clusters, kernel, &cfg), "cudaOccupancyMaxActiveClusters")) != cudaSuccess) return e;
+      if (max_clusters < 1) return cuda_note(cudaErrorLaunchOutOfResources, "no cluster of this size fits the device");
       known[key] = max_clusters;
     }
   }
@@ -760,7 +749,7 @@ static cudaError_t cluster_launch_one(const ClArgs& a, const ClPlan& p, cudaStre
   const int64_t clusters = rows < max_clusters ? rows : max_clusters;
   cfg.gridDim = dim3((unsigned)(clusters * p.cluster));
   cfg.numAttrs = 2;
-  e = cudaLaunchKernelEx(&cfg, kernel, a);
+  e = cuda_note(cudaLaunchKernelEx(&cfg, kernel, a), "cudaLaunchKernelEx (cluster kernel)");
   return e != cudaSuccess ? e : cudaGetLastError();
 }
 

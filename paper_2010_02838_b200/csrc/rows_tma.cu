@@ -39,6 +39,7 @@ constexpr int kSegPerThread = 2;       // 16-byte segments per consumer thread p
 constexpr int kMaxConsumerWarps = 16;
 constexpr uint32_t kBulkPieceBytes = 32768;
 constexpr unsigned long long kWaitLimitNs = 2000000000ull;  // bounded waits: 2 s, then CODISTILL_DEV_TIMEOUT
+constexpr unsigned long long kDrainLimitNs = 50000000ull;   // per barrier when a producer leaves: 50 ms
 
 struct TmaCfg {
   int consumer_warps;  // 8 (two CTAs per SM) or 16 (one CTA per SM)
@@ -77,33 +78,20 @@ struct Ctrl {  // lives at the start of dynamic shared memory
 static_assert(sizeof(Ctrl) <= kCtrlBytes - kZeroBytes, "control block fits its slot");
 
 // Wait for a phase of an mbarrier, but never for ever: after kWaitLimitNs the CTA-wide abort flag
-// and the device status are set and every later wait returns at once (results are then invalid).
-// The polling loop is kept out of line so that the callers' code stays compact.
-__device__ __noinline__ void wait_slow(uint64_t* bar, uint32_t parity, Ctrl* ctrl, WsHeader* hdr) {
-  volatile int* abort_flag = &ctrl->abort_flag;
-  uint32_t polls = 0;
-  unsigned long long t0 = 0;
-  // The producer warps wait most of the time and have slack (ring stages, row pieces ahead): they
-  // back off between polls, so that their polling does not take issue slots from the consumers.
-  const bool producer = threadIdx.x < kProducerThreads;
-  while (!mbar_try_wait(bar, parity)) {
-    if (producer) __nanosleep(128);
-    if ((++polls & 0x3FFu) == 0) {
-      if (*abort_flag) return;
-      const unsigned long long now = global_timer_ns();
-      if (t0 == 0) {
-        t0 = now;
-      } else if (now - t0 > kWaitLimitNs) {
-        *abort_flag = 1;
-        atomicOr(&hdr->status, CODISTILL_DEV_TIMEOUT);
-        return;
-      }
-    }
-  }
-}
+// and the device status are set and every later wait returns early (results are then invalid).  The
+// producer warps wait most of the time and have slack (ring stages, row pieces ahead): they back off
+// between polls, so that their polling does not take issue slots from the consumers.
 __device__ __forceinline__ void wait_bounded(uint64_t* bar, uint32_t parity, Ctrl* ctrl, WsHeader* hdr) {
   if (mbar_try_wait(bar, parity)) return;
-  wait_slow(bar, parity, ctrl, hdr);
+  mbar_wait_limited(bar, parity, &ctrl->abort_flag, &hdr->status, CODISTILL_DEV_TIMEOUT, kWaitLimitNs, true,
+                    threadIdx.x < kProducerThreads);
+}
+// Last wait of a producer warp on a barrier it armed: also after an abort the copies that complete on it
+// get one further, shorter interval to land, so that the CTA does not end with a copy into its shared
+// memory still in flight.
+__device__ __forceinline__ void wait_drain(uint64_t* bar, uint32_t parity, Ctrl* ctrl, WsHeader* hdr) {
+  if (mbar_try_wait(bar, parity)) return;
+  mbar_wait_limited(bar, parity, &ctrl->abort_flag, &hdr->status, CODISTILL_DEV_TIMEOUT, kDrainLimitNs, false, true);
 }
 
 // Block reductions among the NCW * 32 consumer threads (one named barrier each).
@@ -408,7 +396,7 @@ rows_tma_kernel(const __grid_constant__ KArgs a, const TmaCfg cfg) {
     if (lane == 0) bulk_wait_all_groups();  // zero rows are written
     // Before leaving, make sure no copy armed by this warp is still in flight (bounded).
     if (v >= 1)
-      for (int k = 0; k < n_pieces; ++k) wait_bounded(&ctrl->own_full[k], (v - 1) & 1, ctrl, a.hdr);
+      for (int k = 0; k < n_pieces; ++k) wait_drain(&ctrl->own_full[k], (v - 1) & 1, ctrl, a.hdr);
   } else if (warp == 1) {
     // ============================== peer producer ==============================
     uint32_t q = 0;          // ring items issued so far
@@ -439,7 +427,7 @@ rows_tma_kernel(const __grid_constant__ KArgs a, const TmaCfg cfg) {
     }
     for (uint32_t i = 0; i < (uint32_t)n_stage && i < q; ++i) {
       const uint32_t qi = q - 1 - i;
-      wait_bounded(&ctrl->ring_full[qi % n_stage], (qi / n_stage) & 1, ctrl, a.hdr);
+      wait_drain(&ctrl->ring_full[qi % n_stage], (qi / n_stage) & 1, ctrl, a.hdr);
     }
   } else {
     // ============================== consumer warps ==============================
@@ -648,7 +636,7 @@ rows_tma_kernel(const __grid_constant__ KArgs a, const TmaCfg cfg) {
       const uint32_t spec_y = (((seg_y % kSegPerChunk) % kConsumers) == tid) ? 1u << (seg_y / kSegPerChunk) : 0u;
       const uint32_t spec_a = (seg_a >= 0 && ((seg_a % kSegPerChunk) % kConsumers) == tid) ? 1u << (seg_a / kSegPerChunk) : 0u;
       const int u_y = (seg_y % kSegPerChunk) / kConsumers, u_a = seg_a >= 0 ? (seg_a % kSegPerChunk) / kConsumers : 0;
-      const bool lean_ok = with_term && a.want_flags && g_img != nullptr;
+      const bool lean_ok = with_term && g_img != nullptr;   // without counters seg_a is -1: the agreement maxima are kept but never read
       float2 dist2b = make_float2(0.f, 0.f);
       const uint32_t tid16 = (uint32_t)tid * 16u;
 

@@ -74,6 +74,18 @@ def test_all_models_call_every_cluster_size(cluster_size, n, C, dtype):
                     temperature=T)
 
 
+@pytest.mark.parametrize("n", [5, 6, 7])
+@pytest.mark.parametrize("dtype", ["f32", "bf16"])
+def test_plain_mse_with_four_to_six_peers_stays_on_a_long_row_kernel(n, dtype):
+    """The staged and direct-load MSE kernels are built for 0-3 and 7 peers; the peer counts between are
+    served by the cluster-resident kernel, not by the one-CTA-per-row fallback."""
+    rows, C = 300, 9001 if dtype == "bf16" else 4099
+    models, labels, mask = rand_models(43 * n, rows, C, n, dtype)
+    for pr in (cb.PEERS_PAIRWISE_MEAN, cb.PEERS_MEAN_TARGET):
+        compare(models[0], models[1:], labels, mask, alpha=0.9, label_smoothing=0.05, peer_reduce=pr,
+                reduction=cb.REDUCE_SUM, expect_regime="cluster")
+
+
 @pytest.mark.parametrize("dtype", ["f32", "bf16"])
 def test_maxima_on_range_boundaries(cluster_size, dtype):
     """Equal maxima planted in the last column of one CTA's range and the first column of the next, on the

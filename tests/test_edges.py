@@ -181,3 +181,16 @@ def test_host_buffer_entry_point(monkeypatch, regime, dist):
     np.testing.assert_allclose(h_row.numpy(), ref.row_loss, rtol=2e-3)
     g = synth.bf16_bits_to_f32(h_grad.numpy().view(np.uint16)).astype(np.float64)
     assert np.abs(g - ref.grad).max() <= 2e-3
+
+
+def test_expired_wait_sets_the_status_bit_and_the_context_stays_usable():
+    """A wait on an asynchronous copy that runs out of time ends in CODISTILL_DEV_TIMEOUT and a normal
+    kernel exit.  The diagnostic call waits 1 ms on a barrier nothing completes (no copy is involved);
+    an ordinary call right after it gives the oracle's result."""
+    status = cb.selftest_bounded_wait(1_000_000)
+    torch.cuda.synchronize()
+    assert int(status.item()) == cb.DEV_TIMEOUT
+    own, peers, labels = rand_inputs(3, 12, 8192, 2, "bf16")
+    compare(own, peers, labels, None, alpha=1.0, reduction=cb.REDUCE_SUM, expect_regime="tma")
+    with pytest.raises(cb.CodistillError):
+        cb.selftest_bounded_wait(10 ** 9)     # limits beyond 100 ms are refused on the host

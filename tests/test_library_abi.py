@@ -1,4 +1,4 @@
-"""The C-ABI library builds, loads and exports every symbol declared in include/codistill.h
+"""The C-ABI library builds, loads and exports every symbol declared in include/*.h
 (no compute calls: runs without a GPU)."""
 import ctypes
 import os
@@ -19,9 +19,13 @@ def lib():
 
 
 def declared_functions():
-    text = open(os.path.join(ROOT, "include", "codistill.h")).read()
-    text = re.sub(r"/\*.*?\*/", "", text, flags=re.S)
-    return sorted(set(re.findall(r"\b(codistill_[a-z_0-9]+)\s*\(", text)))
+    names = set()
+    inc = os.path.join(ROOT, "include")
+    for header in sorted(os.listdir(inc)):
+        text = open(os.path.join(inc, header)).read()
+        text = re.sub(r"/\*.*?\*/", "", text, flags=re.S)
+        names |= set(re.findall(r"\b(codistill_[a-z_0-9]+)\s*\(", text))
+    return sorted(names)
 
 
 def test_exports_every_declared_symbol(lib):

@@ -53,3 +53,14 @@ def test_two_ranks_independent_batches_and_max_time():
     assert first0 != first1 and loss0 != loss1            # different seeds: different batches
     assert ms0 == ms1 == 2.0                              # max over ranks
     assert v0 == v1 == 2 * 64 / 2e-3                      # whole-job rows/s
+
+
+def test_bench_starts_one_rank_per_gpu_when_asked_outside_a_launcher():
+    """`bench.py --gpus N` run as a plain script re-launches itself under torchrun with N local ranks."""
+    sys.path.insert(0, ROOT)
+    import bench
+    cmd = bench.torchrun_command(["--gpus", "4", "--steps", "7"], 4, port=29431)
+    assert cmd[:3] == [sys.executable, "-m", "torch.distributed.run"]
+    assert "--nproc-per-node=4" in cmd and "--nnodes=1" in cmd
+    assert cmd[cmd.index("--master-addr") + 1] == "127.0.0.1" and cmd[cmd.index("--master-port") + 1] == "29431"
+    assert cmd[-5:] == [os.path.join(ROOT, "bench.py"), "--gpus", "4", "--steps", "7"]
