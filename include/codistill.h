@@ -76,8 +76,7 @@ enum { CODISTILL_REDUCE_MEAN_VALID = 0, CODISTILL_REDUCE_SUM = 1 };
 /* bits OR-ed into *dev_status by the kernels */
 enum {
   CODISTILL_DEV_BAD_LABEL = 1, /* a valid row had a label outside [0, classes); that row was treated as masked */
-  CODISTILL_DEV_TIMEOUT = 2,   /* a bounded wait on an asynchronous copy expired; outputs are not to be trusted */
-  CODISTILL_DEV_ASSERT = 4     /* an internal consistency check failed */
+  CODISTILL_DEV_TIMEOUT = 2    /* a bounded wait on an asynchronous copy expired; outputs are not to be trusted */
 };
 
 #define CODISTILL_MAX_PEERS 31 /* n <= 32 */

@@ -20,7 +20,7 @@ F32, BF16 = 0, 1
 DIST_MSE_LOGITS, DIST_KL_SOFTMAX, DIST_MSE_CENTRED = 0, 1, 2
 PEERS_PAIRWISE_MEAN, PEERS_MEAN_TARGET = 0, 1
 REDUCE_MEAN_VALID, REDUCE_SUM = 0, 1
-DEV_BAD_LABEL, DEV_TIMEOUT, DEV_ASSERT = 1, 2, 4
+DEV_BAD_LABEL, DEV_TIMEOUT = 1, 2
 MAX_PEERS = 31
 STATIC_MAX_ROWS = 65536
 ERR_CUDA = 6

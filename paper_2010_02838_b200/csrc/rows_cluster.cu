@@ -25,6 +25,7 @@
 // averaged peer logits (mean target, single-model call only) takes the statistics of that average
 // as one more tensor in pass A.
 #include <cooperative_groups.h>
+#include <stdio.h>
 #include <stdlib.h>
 #include <string.h>
 
@@ -44,9 +45,8 @@ namespace codistill {
 
 constexpr int kClThreads = 256;
 constexpr int kClWarps = kClThreads / 32;
-constexpr int kClMaxRecs = 3;                      // pass-A records per warp (its range spans at most that many tensors)
 constexpr int kClMaxCluster = 16;
-constexpr int kClCtrlBytes = 4096;
+constexpr int kClCtrlBytes = 12288;
 constexpr uint32_t kClCopyPiece = 32768;
 constexpr unsigned long long kClWaitLimitNs = 2000000000ull;   // bounded waits: 2 s, then CODISTILL_DEV_TIMEOUT
 constexpr unsigned long long kClDrainLimitNs = 50000000ull;    // last wait of an aborted CTA: 50 ms
@@ -54,18 +54,16 @@ constexpr unsigned long long kClDrainLimitNs = 50000000ull;    // last wait of a
 // what one warp found in a sub-range of one tensor
 struct ClRec { float m; int seg; float S, sum_z, S_T; int tensor; };
 // what one CTA found in its range of one tensor
-struct ClPart { float m; int col; float S, sum_z, S_T, zy; int has_y; int pad; };
+struct ClPart { float m; int col; float S, sum_z, S_T, zy; };   // zy: the label's logit if it lies in the range, else 0
 // statistics of a whole row of one tensor
 struct ClStat { float m, S, sum_z, S_T, zy; int col; };
 
 struct ClCtrl {
-  uint64_t full;                           // bulk copies of the current row have landed
+  uint64_t full[kClMax];                   // bulk copies of tensor i's range of the current row have landed
   int abort_flag;
-  int nrec[kClWarps];
-  ClRec rec[kClWarps][kClMaxRecs];
-  ClRec rec_mean[kClWarps];                // KL mean target: statistics of the averaged peers
-  ClPart part[2][kClMax + 1];              // [row parity][tensor]; slot n: the averaged peers
-  float dpart[2][kClMax + 1];              // distance partial sums per model; slot kClMax: sum_j z'_j^2
+  ClRec rec[kClWarps][kClMax + 1];         // pass A: what warp w found in its share of tensor i (slot n: the averaged peers)
+  ClPart gather[2][kClMaxCluster][kClMax + 1];   // [row parity][CTA of the cluster][tensor]: written by that CTA into every CTA
+  float dgather[2][kClMaxCluster][kClMax + 1];   // CTA 0: distance partial sums [parity][CTA][model]; slot kClMax: sum_j z'_j^2
   float dwarp[kClWarps][kClMax + 1];
   ClStat stat[kClMax + 1];                 // current row, combined over the cluster
   ClStat pend[2][kClMax + 1];              // CTA 0: statistics of the rows whose loss is still to be written
@@ -78,7 +76,7 @@ static_assert(sizeof(ClCtrl) <= kClCtrlBytes, "control block fits its slot");
 // device status are set and later waits return early (results are then invalid, control flow stays uniform).
 __device__ __forceinline__ void cl_wait(uint64_t* bar, uint32_t parity, ClCtrl* ctrl, WsHeader* hdr) {
   if (mbar_try_wait(bar, parity)) return;
-  mbar_wait_limited(bar, parity, &ctrl->abort_flag, &hdr->status, CODISTILL_DEV_TIMEOUT, kClWaitLimitNs, true, false);
+  mbar_wait_limited(bar, parity, &ctrl->abort_flag, &hdr->status, CODISTILL_DEV_TIMEOUT, kClWaitLimitNs, true, true);
 }
 
 // exp((z - m) / T) for a pair of columns; l2eT = log2(e) / T
@@ -97,22 +95,31 @@ __device__ __forceinline__ float exp_nat1(float x) {
   if constexpr (sizeof(T) == 4) return expf(x); else return ex2_approx(x * kLog2e);
 }
 
-// Running statistics of one thread over its segments of one tensor (visited in rising order).
+// Running statistics of one thread over its segments of one tensor (visited in rising order); one
+// partial sum per pair position of a segment, so that the additions of a segment do not form a chain.
+template <int H>
 struct ClAcc {
   float best;       // finite start value, so that the first rescale is exp2(-huge) = 0 and never NaN
   int best_seg;
-  float2 s2, t2, zs2;
-  __device__ void reset() { best = -3.0e38f; best_seg = 0x7fffffff; s2 = make_float2(0.f, 0.f); t2 = s2; zs2 = s2; }
+  float2 s2[H], t2[H], zs2[H];
+  __device__ __forceinline__ void reset() {
+    best = -3.0e38f;
+    best_seg = 0x7fffffff;
+#pragma unroll
+    for (int h = 0; h < H; ++h) { s2[h] = make_float2(0.f, 0.f); t2[h] = s2[h]; zs2[h] = s2[h]; }
+  }
 };
 
-template <typename T, bool TEMP>
-__device__ __forceinline__ void cl_raise(ClAcc& acc, float fm, int s, float inv_T) {
+template <typename T, bool TEMP, int H>
+__device__ __forceinline__ void cl_raise(ClAcc<H>& acc, float fm, int s, float inv_T) {
   if (fm > acc.best) {
     const float sc = rescale_exp2<T>((acc.best - fm) * kLog2e);
-    acc.s2 = __fmul2_rn(acc.s2, make_float2(sc, sc));
+#pragma unroll
+    for (int h = 0; h < H; ++h) acc.s2[h] = __fmul2_rn(acc.s2[h], make_float2(sc, sc));
     if constexpr (TEMP) {
       const float st = rescale_exp2<T>((acc.best - fm) * (kLog2e * inv_T));
-      acc.t2 = __fmul2_rn(acc.t2, make_float2(st, st));
+#pragma unroll
+      for (int h = 0; h < H; ++h) acc.t2[h] = __fmul2_rn(acc.t2[h], make_float2(st, st));
     }
     acc.best = fm;
     acc.best_seg = s;
@@ -121,7 +128,7 @@ __device__ __forceinline__ void cl_raise(ClAcc& acc, float fm, int s, float inv_
 
 // one whole segment (all of its columns lie inside the row)
 template <typename T, bool TEMP>
-__device__ __forceinline__ void cl_sweep_seg(ClAcc& acc, const uint4& raw, int s, float inv_T) {
+__device__ __forceinline__ void cl_sweep_seg(ClAcc<SegOps<T>::H>& acc, const uint4& raw, int s, float inv_T, bool need_z) {
   constexpr int H = SegOps<T>::H;
   cl_raise<T, TEMP>(acc, SegOps<T>::to_float(SegOps<T>::fold(raw)), s, inv_T);
   const float2 l2e2 = make_float2(kLog2e, kLog2e);
@@ -130,15 +137,19 @@ __device__ __forceinline__ void cl_sweep_seg(ClAcc& acc, const uint4& raw, int s
   SegOps<T>::unpack2(raw, z2);
 #pragma unroll
   for (int h = 0; h < H; ++h) {
-    acc.s2 = __fadd2_rn(acc.s2, exp_shift2<T>(z2[h], acc.best, l2e2, nmk));
-    acc.zs2 = __fadd2_rn(acc.zs2, z2[h]);
-    if constexpr (TEMP) acc.t2 = __fadd2_rn(acc.t2, exp_temp2<T>(z2[h], acc.best, inv_T, kLog2e * inv_T));
+    acc.s2[h] = __fadd2_rn(acc.s2[h], exp_shift2<T>(z2[h], acc.best, l2e2, nmk));
+    if constexpr (TEMP) acc.t2[h] = __fadd2_rn(acc.t2[h], exp_temp2<T>(z2[h], acc.best, inv_T, kLog2e * inv_T));
+  }
+  if (need_z) {   // the sum of the logits: label smoothing and the centred distance only
+#pragma unroll
+    for (int h = 0; h < H; ++h) acc.zs2[h] = __fadd2_rn(acc.zs2[h], z2[h]);
   }
 }
 
 // a ragged segment (first or last of the row image): only the columns inside the row count
+// (accumulators in and out by value, so that the caller's copy stays in registers)
 template <typename T, bool TEMP>
-__device__ __noinline__ void cl_sweep_edge(ClAcc& acc, uint4 raw, int s, int head, int64_t C, float inv_T) {
+__device__ __noinline__ ClAcc<SegOps<T>::H> cl_sweep_edge(ClAcc<SegOps<T>::H> acc, uint4 raw, int s, int head, int64_t C, float inv_T) {
   constexpr int V = SegOps<T>::V;
   float z[V];
   SegOps<T>::unpack(raw, z);
@@ -155,27 +166,148 @@ __device__ __noinline__ void cl_sweep_edge(ClAcc& acc, uint4 raw, int s, int hea
   for (int e = 0; e < V; ++e) {
     const int64_t c = (int64_t)s * V - head + e;
     if (c >= 0 && c < C) {
-      acc.s2.x += exp_shift2<T>(make_float2(z[e], z[e]), acc.best, l2e2, nmk).x;
-      acc.zs2.x += z[e];
-      if constexpr (TEMP) acc.t2.x += exp_temp2<T>(make_float2(z[e], z[e]), acc.best, inv_T, kLog2e * inv_T).x;
+      acc.s2[0].x += exp_shift2<T>(make_float2(z[e], z[e]), acc.best, l2e2, nmk).x;
+      acc.zs2[0].x += z[e];
+      if constexpr (TEMP) acc.t2[0].x += exp_temp2<T>(make_float2(z[e], z[e]), acc.best, inv_T, kLog2e * inv_T).x;
     }
   }
+  return acc;
 }
 
 // Reduces the lanes' accumulators of one sub-range to one record (all lanes take part).
-template <typename T, bool TEMP>
-__device__ __forceinline__ ClRec cl_warp_record(const ClAcc& acc, int tensor, float inv_T) {
+template <typename T, bool TEMP, int H>
+__device__ __forceinline__ ClRec cl_warp_record(const ClAcc<H>& acc, int tensor, float inv_T) {
   const unsigned key = float_order_key(acc.best + 0.f);   // -0 is folded onto +0: they tie
   const unsigned key_w = __reduce_max_sync(0xffffffffu, key);
+  float s_t = 0.f, z_t = 0.f, t_t = 0.f;
+#pragma unroll
+  for (int h = 0; h < H; ++h) { s_t += acc.s2[h].x + acc.s2[h].y; z_t += acc.zs2[h].x + acc.zs2[h].y; t_t += acc.t2[h].x + acc.t2[h].y; }
   ClRec r;
   r.seg = (int)__reduce_min_sync(0xffffffffu, key == key_w ? (unsigned)acc.best_seg : 0x7fffffffu);
   r.m = float_from_order_key(key_w);
-  r.S = warp_sum((acc.s2.x + acc.s2.y) * rescale_exp2<T>((acc.best - r.m) * kLog2e));
-  r.sum_z = warp_sum(acc.zs2.x + acc.zs2.y);
+  r.S = warp_sum(s_t * rescale_exp2<T>((acc.best - r.m) * kLog2e));
+  r.sum_z = warp_sum(z_t);
   r.S_T = 0.f;
-  if constexpr (TEMP) r.S_T = warp_sum((acc.t2.x + acc.t2.y) * rescale_exp2<T>((acc.best - r.m) * (kLog2e * inv_T)));
+  if constexpr (TEMP) r.S_T = warp_sum(t_t * rescale_exp2<T>((acc.best - r.m) * (kLog2e * inv_T)));
   r.tensor = tensor;
   return r;
+}
+
+// Combines partial results (one per lane; lanes without one pass m = -3e38, S = 0, pos = INT_MAX) across
+// the warp: the maximum, the lowest position among those that attain it, the sums rescaled to it.
+template <typename T>
+__device__ __forceinline__ void cl_warp_combine(float& m, int& pos, float& S, float& sum_z, float& S_T, bool temp, float inv_T) {
+  const unsigned key = float_order_key(m + 0.f);
+  const unsigned key_m = __reduce_max_sync(0xffffffffu, key);
+  const float mm = float_from_order_key(key_m);
+  pos = (int)__reduce_min_sync(0xffffffffu, key == key_m ? (unsigned)pos : 0x7fffffffu);
+  S = warp_sum(S * rescale_exp2<T>((m - mm) * kLog2e));
+  if (temp) S_T = warp_sum(S_T * rescale_exp2<T>((m - mm) * (kLog2e * inv_T)));
+  sum_z = warp_sum(sum_z);
+  m = mm;
+}
+
+// What pass B needs of the row statistics (registers), and its running sums.
+template <int N, int NS>
+struct ClColCtx {
+  float mi[N], cpi[N], cmi[N];   // per model: maximum, w / S, centred distance: -(class mean - average class mean of the models)
+  float cti[NS], lsi[NS];        // KL: 1 / S_T and log S_T (slot N: the averaged peers)
+  float mb;                      // KL mean target: maximum of the averaged peers
+  float cd, cq, cy, ckl, inv_T;
+  bool t_one, centred;
+  int y;
+};
+template <int NOUT>
+struct ClColAcc {
+  float2 dist2[NOUT], qs2;
+};
+
+// Two neighbouring columns c, c + 1 of the n models (zc): distance terms into `acc`, gradient pairs of the
+// requested models into gc.  `lab`: c or c + 1 may be the label column.  RAGGED: a column of the pair may lie
+// outside the row (in2 = 1 / 0 per column); such columns contribute nothing.
+template <typename T, int N, int MODE, bool ALL, bool RAGGED, int NS>
+__device__ __forceinline__ void cl_column2(const ClColCtx<N, NS>& x, ClColAcc<ALL ? N : 1>& acc, const float2 (&zc)[N],
+                                           float2 (&gc)[ALL ? N : 1], int64_t c, bool lab, float2 in2) {
+  constexpr int NOUT = ALL ? N : 1;
+  float2 ncq = make_float2(-x.cq, -x.cq);
+  if (lab) ncq = make_float2((c == (int64_t)x.y) ? -(x.cq + x.cy) : -x.cq, (c + 1 == (int64_t)x.y) ? -(x.cq + x.cy) : -x.cq);
+  auto inside = [&](float2 v) { if constexpr (RAGGED) return __fmul2_rn(v, in2); else return v; };
+  const float2 l2e2 = make_float2(kLog2e, kLog2e);
+  if constexpr (MODE == kClMse) {
+    // z'_i = z_i - mean_j z_j, for the centred distance on z_i - (class mean of model i); x.cmi[i] holds
+    // -(class mean_i - mean_j class mean_j), so one addition per model centres both ways
+    float2 zp[N], mu = zc[0];
+#pragma unroll
+    for (int i = 1; i < N; ++i) mu = __fadd2_rn(mu, zc[i]);
+    mu = __fmul2_rn(mu, make_float2(-1.f / (float)N, -1.f / (float)N));
+#pragma unroll
+    for (int i = 0; i < N; ++i) zp[i] = __fadd2_rn(zc[i], mu);
+    if (x.centred) {
+#pragma unroll
+      for (int i = 0; i < N; ++i) zp[i] = __fadd2_rn(zp[i], make_float2(x.cmi[i], x.cmi[i]));
+    }
+    if constexpr (RAGGED) {
+#pragma unroll
+      for (int i = 0; i < N; ++i) zp[i] = __fmul2_rn(zp[i], in2);
+    }
+    if constexpr (!ALL) {   // sum_j z'_j^2 of the pairwise form (with every model's output it is the sum of their distance sums)
+      float2 q = make_float2(0.f, 0.f);
+#pragma unroll
+      for (int i = 0; i < N; ++i) q = __ffma2_rn(zp[i], zp[i], q);
+      acc.qs2 = __fadd2_rn(acc.qs2, q);
+    }
+#pragma unroll
+    for (int i = 0; i < NOUT; ++i) {
+      const float nm = -x.mi[i] * kLog2e;
+      const float2 e = exp_shift2<T>(zc[i], x.mi[i], l2e2, make_float2(nm, nm));
+      gc[i] = __ffma2_rn(e, make_float2(x.cpi[i], x.cpi[i]), __ffma2_rn(make_float2(x.cd, x.cd), zp[i], ncq));
+      acc.dist2[i] = __ffma2_rn(zp[i], zp[i], acc.dist2[i]);
+    }
+  } else if constexpr (MODE == kClKlPairwise) {
+    float2 t[N], lt[N], Q = make_float2(0.f, 0.f), E = make_float2(0.f, 0.f);
+#pragma unroll
+    for (int i = 0; i < N; ++i) {
+      float2 e1 = make_float2(0.f, 0.f);
+      if (x.t_one || i < NOUT) {
+        const float nm = -x.mi[i] * kLog2e;
+        e1 = exp_shift2<T>(zc[i], x.mi[i], l2e2, make_float2(nm, nm));
+      }
+      const float2 et = x.t_one ? e1 : exp_temp2<T>(zc[i], x.mi[i], x.inv_T, kLog2e * x.inv_T);
+      t[i] = inside(__fmul2_rn(et, make_float2(x.cti[i], x.cti[i])));
+      const float2 d = __fadd2_rn(zc[i], make_float2(-x.mi[i], -x.mi[i]));
+      const float2 l = __ffma2_rn(d, make_float2(x.inv_T, x.inv_T), make_float2(-x.lsi[i], -x.lsi[i]));
+      lt[i] = make_float2(fmaxf(l.x, -3.0e38f), fmaxf(l.y, -3.0e38f));   // log t_i, kept finite: 0 * log 0 = 0
+      Q = __fadd2_rn(Q, t[i]);
+      E = __ffma2_rn(t[i], lt[i], E);
+      if (i < NOUT) gc[i] = __ffma2_rn(e1, make_float2(x.cpi[i], x.cpi[i]), ncq);
+    }
+    const float2 nQ = make_float2(-Q.x, -Q.y);
+#pragma unroll
+    for (int i = 0; i < NOUT; ++i) {
+      gc[i] = __ffma2_rn(make_float2(x.ckl, x.ckl), __ffma2_rn(make_float2((float)N, (float)N), t[i], nQ), gc[i]);
+      acc.dist2[i] = __fadd2_rn(acc.dist2[i], __ffma2_rn(nQ, lt[i], E));   // sum_{j != i} t_j (log t_j - log t_i)
+    }
+  } else {
+    // KL to the softmax of the averaged peers: t = softmax(zbar / T), p^T = softmax(z_0 / T)
+    const float inv_P = 1.f / (float)(N - 1);
+    float2 zb = make_float2(0.f, 0.f);
+#pragma unroll
+    for (int j = 1; j < N; ++j) zb = __fadd2_rn(zb, zc[j]);
+    zb = __fmul2_rn(zb, make_float2(inv_P, inv_P));
+    const float nm = -x.mi[0] * kLog2e;
+    const float2 e1 = exp_shift2<T>(zc[0], x.mi[0], l2e2, make_float2(nm, nm));
+    const float2 eT = x.t_one ? e1 : exp_temp2<T>(zc[0], x.mi[0], x.inv_T, kLog2e * x.inv_T);
+    const float2 pT = __fmul2_rn(eT, make_float2(x.cti[0], x.cti[0]));
+    const float2 x0 = __fadd2_rn(zc[0], make_float2(-x.mi[0], -x.mi[0]));
+    const float2 lp = __ffma2_rn(x0, make_float2(x.inv_T, x.inv_T), make_float2(-x.lsi[0], -x.lsi[0]));
+    const float2 tb = inside(__fmul2_rn(exp_temp2<T>(zb, x.mb, x.inv_T, kLog2e * x.inv_T), make_float2(x.cti[N], x.cti[N])));
+    const float2 xb = __fadd2_rn(zb, make_float2(-x.mb, -x.mb));
+    const float2 lb = __ffma2_rn(xb, make_float2(x.inv_T, x.inv_T), make_float2(-x.lsi[N], -x.lsi[N]));
+    const float2 dl = make_float2(fmaxf(lb.x, -3.0e38f) - fmaxf(lp.x, -3.0e38f), fmaxf(lb.y, -3.0e38f) - fmaxf(lp.y, -3.0e38f));
+    gc[0] = __ffma2_rn(make_float2(x.ckl, x.ckl), __fadd2_rn(pT, make_float2(-tb.x, -tb.y)),
+                       __ffma2_rn(e1, make_float2(x.cpi[0], x.cpi[0]), ncq));
+    acc.dist2[0] = __ffma2_rn(tb, dl, acc.dist2[0]);
+  }
 }
 
 // ------------------------------------------------------------------ the kernel
@@ -189,6 +321,7 @@ __global__ void __launch_bounds__(kClThreads, 2) rows_cluster_kernel(const __gri
   constexpr bool KLM = MODE == kClKlMeanTarget;
   constexpr int NOUT = ALL ? N : 1;
   constexpr int NSTAT = KLM ? N + 1 : N;
+  constexpr int NS = KL ? NSTAT : 1;
   constexpr int NW = kClWarps, NT = kClThreads;
   static_assert(!(KLM && ALL), "the mean-target KL distance is a single-model form");
   static_assert(N >= 2 && N <= kClMax, "tensor count");
@@ -204,9 +337,10 @@ __global__ void __launch_bounds__(kClThreads, 2) rows_cluster_kernel(const __gri
   const float inv_C = 1.f / (float)C;
   const float inv_T = KL ? 1.f / a.temperature : 1.f;
   const bool t_one = !KL || a.temperature == 1.f;
+  const bool need_z = a.eps != 0.f || a.centred != 0;   // sum_c z_c enters the smoothed task loss and the class means
 
   if (tid == 0) {
-    mbar_init(&ctrl->full, 1);
+    for (int i = 0; i < N; ++i) mbar_init(&ctrl->full[i], 1);
     ctrl->abort_flag = 0;
     mbar_init_fence();
   }
@@ -221,11 +355,16 @@ __global__ void __launch_bounds__(kClThreads, 2) rows_cluster_kernel(const __gri
     w = 1.f / (float)(nv > 1 ? nv : 1);
   }
   constexpr float kRatio = (float)N / (float)(N - 1);                 // z_i - zbar_(-i) = kRatio * z'_i
-  const float cd = w * a.alpha * (2.f * inv_C) * kRatio;               // z'_i -> w alpha dD_i/dz_i      (MSE)
-  const float cq = w * a.eps * inv_C;
-  const float cy = w * (1.f - a.eps);
-  const float ckl = KLM ? w * a.alpha * a.temperature                  // (p^T - t) -> w alpha dD/dz
-                        : w * a.alpha * a.temperature / (float)(N - 1);  // (n t_i - Q) -> w alpha dD_i/dz_i
+  ClColCtx<N, NS> cx;
+  cx.cd = w * a.alpha * (2.f * inv_C) * kRatio;                        // z'_i -> w alpha dD_i/dz_i      (MSE)
+  cx.cq = w * a.eps * inv_C;
+  cx.cy = w * (1.f - a.eps);
+  cx.ckl = KLM ? w * a.alpha * a.temperature                           // (p^T - t) -> w alpha dD/dz
+               : w * a.alpha * a.temperature / (float)(N - 1);         // (n t_i - Q) -> w alpha dD_i/dz_i
+  cx.inv_T = inv_T;
+  cx.t_one = t_one;
+  cx.centred = a.centred != 0;
+  cx.mb = 0.f;
   const int seg_begin = rank * a.spc;
 
   auto row_is_valid = [&](long long r) {
@@ -238,7 +377,10 @@ __global__ void __launch_bounds__(kClThreads, 2) rows_cluster_kernel(const __gri
     const int64_t lr = r - a.row_begin;
     const RowGeom g = row_geom<T>(lr, a.row_stride, C);
     const int seg_end = min(seg_begin + a.spc, g.n_seg);
-    if (seg_end <= seg_begin) { mbar_arrive(&ctrl->full); return; }
+    if (seg_end <= seg_begin) {
+      for (int i = 0; i < N; ++i) mbar_arrive(&ctrl->full[i]);
+      return;
+    }
     const uint32_t begin = (uint32_t)seg_begin * 16u, end = (uint32_t)seg_end * 16u;
     // The last row of the whole call may end inside a segment that reaches past the tensor: that
     // segment is fetched element by element, whole-segment copies stop before it.
@@ -247,34 +389,25 @@ __global__ void __launch_bounds__(kClThreads, 2) rows_cluster_kernel(const __gri
     const uint32_t copy_end = clip ? (valid_end & ~15u) : end;
     const uint32_t bytes = copy_end > begin ? copy_end - begin : 0u;
     const int64_t img_off = (lr * a.row_stride - g.head) * ES;   // image start relative to the tensor
-    if (clip) {
-#pragma unroll 1
-      for (int i = 0; i < N; ++i) {
-        const char* src = reinterpret_cast<const char*>(a.model[i]) + img_off;
-        char* dst = slices + (size_t)i * a.slice_bytes - begin;
-        for (uint32_t o = copy_end > begin ? copy_end : begin; o < valid_end; o += ES)
-          *reinterpret_cast<T*>(dst + o) = *reinterpret_cast<const T*>(src + o);
-      }
-    }
-    mbar_arrive_expect_tx(&ctrl->full, bytes * (uint32_t)N);
 #pragma unroll 1
     for (int i = 0; i < N; ++i) {
-      const char* src = reinterpret_cast<const char*>(a.model[i]) + img_off + begin;
+      const char* src = reinterpret_cast<const char*>(a.model[i]) + img_off;
       char* dst = slices + (size_t)i * a.slice_bytes;
+      if (clip) {
+        for (uint32_t o = copy_end > begin ? copy_end : begin; o < valid_end; o += ES)
+          *reinterpret_cast<T*>(dst + (o - begin)) = *reinterpret_cast<const T*>(src + o);
+      }
+      mbar_arrive_expect_tx(&ctrl->full[i], bytes);
       for (uint32_t o = 0; o < bytes; o += kClCopyPiece)
-        bulk_g2s(dst + o, src + o, bytes - o < kClCopyPiece ? bytes - o : kClCopyPiece, &ctrl->full);
+        bulk_g2s(dst + o, src + begin + o, bytes - o < kClCopyPiece ? bytes - o : kClCopyPiece, &ctrl->full[i]);
     }
   };
-  // CTA 0: loss and flag word of the pending row with parity `pp`, from the K distance partials.
+  // CTA 0: loss and flag word of the pending row with parity `pp`; every CTA has stored its distance
+  // partial sums into this CTA's dgather before the cluster barrier that precedes this call.
   auto finish_row = [&](int pp) {
     for (int i = warp; i < NOUT; i += NW) {
-      float dv = 0.f, qv = 0.f;
-      if (lane < K) {
-        const float* dp = cluster.map_shared_rank(&ctrl->dpart[pp][0], lane);
-        dv = dp[i];
-        qv = dp[kClMax];
-      }
-      const float dsum = warp_sum(dv), qsum = warp_sum(qv);
+      const float dsum = warp_sum(lane < K ? ctrl->dgather[pp][lane][i] : 0.f);
+      const float qsum = warp_sum(lane < K ? ctrl->dgather[pp][lane][kClMax] : 0.f);
       if (lane == 0) {
         const ClStat st = ctrl->pend[pp][i];
         const long long r = ctrl->pend_row[pp];
@@ -331,42 +464,33 @@ __global__ void __launch_bounds__(kClThreads, 2) rows_cluster_kernel(const __gri
     }
     const int par = v & 1;
     if (tid == 0 && issued != r) { issue_row(r); issued = r; }
-    cl_wait(&ctrl->full, (uint32_t)v & 1u, ctrl, a.hdr);
 
-    // ================= pass A: statistics of this CTA's range, tensor by tensor
-    // The n * nseg (tensor, segment) items are dealt to the warps in equal contiguous shares, so a
-    // warp reduces once per tensor its share touches (at most kClMaxRecs times), not once per tensor.
-    {
-      const int total = N * nseg;
-      int lo = (int)(((long long)warp * total) / NW);
-      const int hi = (int)(((long long)(warp + 1) * total) / NW);
-      int nrec = 0;
-      while (lo < hi) {
-        const int i = lo / nseg;
-        const int q0 = lo - i * nseg;
-        const int q1 = min(hi - i * nseg, nseg);
-        const char* sl = slices + (size_t)i * a.slice_bytes;
-        ClAcc acc;
-        acc.reset();
-        for (int q = q0 + lane; q < q1; q += 32) {
-          const int s = seg_begin + q;
-          const uint4 raw = *reinterpret_cast<const uint4*>(sl + (size_t)q * 16);
-          if (s >= g.seg_lo && s < g.seg_hi) {
-            if (t_one) cl_sweep_seg<T, false>(acc, raw, s, inv_T); else cl_sweep_seg<T, KL>(acc, raw, s, inv_T);
-          } else {
-            if (t_one) cl_sweep_edge<T, false>(acc, raw, s, g.head, C, inv_T); else cl_sweep_edge<T, KL>(acc, raw, s, g.head, C, inv_T);
-          }
+    // ================= pass A: statistics of this CTA's range, tensor by tensor as the copies land
+    // Every warp takes a share of each tensor, so the sweep of tensor i runs while tensors i+1.. are still
+    // in flight.  One lane per warp watches the copy barrier (with back-off): waiting warps take next to no
+    // issue slots from the CTA that shares the SM.
+#pragma unroll 1
+    for (int i = 0; i < N; ++i) {
+      if (lane == 0) cl_wait(&ctrl->full[i], (uint32_t)v & 1u, ctrl, a.hdr);
+      __syncwarp();
+      const char* sl = slices + (size_t)i * a.slice_bytes;
+      ClAcc<H> acc;
+      acc.reset();
+      for (int q = tid; q < nseg; q += NT) {
+        const int s = seg_begin + q;
+        const uint4 raw = *reinterpret_cast<const uint4*>(sl + (size_t)q * 16);
+        if (s >= g.seg_lo && s < g.seg_hi) {
+          if (t_one) cl_sweep_seg<T, false>(acc, raw, s, inv_T, need_z); else cl_sweep_seg<T, KL>(acc, raw, s, inv_T, need_z);
+        } else {
+          acc = t_one ? cl_sweep_edge<T, false>(acc, raw, s, g.head, C, inv_T) : cl_sweep_edge<T, KL>(acc, raw, s, g.head, C, inv_T);
         }
-        const ClRec rec = t_one ? cl_warp_record<T, false>(acc, i, inv_T) : cl_warp_record<T, KL>(acc, i, inv_T);
-        if (lane == 0 && nrec < kClMaxRecs) ctrl->rec[warp][nrec] = rec;
-        ++nrec;
-        lo = i * nseg + q1;
       }
-      if (lane == 0) ctrl->nrec[warp] = nrec < kClMaxRecs ? nrec : kClMaxRecs;
+      const ClRec rec = t_one ? cl_warp_record<T, false>(acc, i, inv_T) : cl_warp_record<T, KL>(acc, i, inv_T);
+      if (lane == 0) ctrl->rec[warp][i] = rec;
     }
     if constexpr (KLM) {
       // statistics of the averaged peer logits zbar = mean_{j >= 1} z_j at temperature T
-      ClAcc acc;
+      ClAcc<H> acc;
       acc.reset();
       const float inv_P = 1.f / (float)(N - 1);
       for (int q = tid; q < nseg; q += NT) {
@@ -398,41 +522,28 @@ __global__ void __launch_bounds__(kClThreads, 2) rows_cluster_kernel(const __gri
 #pragma unroll
         for (int h = 0; h < H; ++h) {
           const float2 e2 = exp_temp2<T>(zb[h], acc.best, inv_T, kLog2e * inv_T);
-          if (in[2 * h]) acc.t2.x += e2.x;
-          if (in[2 * h + 1]) acc.t2.y += e2.y;
+          if (in[2 * h]) acc.t2[h].x += e2.x;
+          if (in[2 * h + 1]) acc.t2[h].y += e2.y;
         }
       }
       const ClRec rec = cl_warp_record<T, true>(acc, N, inv_T);
-      if (lane == 0) ctrl->rec_mean[warp] = rec;
+      if (lane == 0) ctrl->rec[warp][N] = rec;
     }
     __syncthreads();
-    if (tid < NSTAT) {
-      // this CTA's partial result of tensor `tid`: records in rising segment order, a strictly larger
-      // maximum replaces the earlier one, so the first segment that attains the maximum is kept
+    // This CTA's partial result of tensor i, by warp i: one warp's record per lane (the first segment that attains
+    // the maximum is the lowest one among the records that attain it), handed to every CTA of the cluster.
+    for (int i = warp; i < NSTAT; i += NW) {
       float m = -3.0e38f, S = 0.f, sum_z = 0.f, S_T = 0.f;
       int seg = 0x7fffffff;
-      auto take = [&](const ClRec& rc) {
-        const float mn = fmaxf(m, rc.m);
-        const float f_old = rescale_exp2<T>((m - mn) * kLog2e), f_new = rescale_exp2<T>((rc.m - mn) * kLog2e);
-        S = S * f_old + rc.S * f_new;
-        if (!t_one || tid == N) {   // the averaged peers (slot N) carry the tempered sum only
-          S_T = S_T * rescale_exp2<T>((m - mn) * (kLog2e * inv_T)) + rc.S_T * rescale_exp2<T>((rc.m - mn) * (kLog2e * inv_T));
-        }
-        sum_z += rc.sum_z;
-        if (rc.m > m) seg = rc.seg;
-        m = mn;
-      };
-      if (tid < N) {
-        for (int wv = 0; wv < NW; ++wv)
-          for (int k = 0; k < ctrl->nrec[wv]; ++k)
-            if (ctrl->rec[wv][k].tensor == tid) take(ctrl->rec[wv][k]);
-      } else {
-        for (int wv = 0; wv < NW; ++wv) take(ctrl->rec_mean[wv]);
+      if (lane < NW) {
+        const ClRec rc = ctrl->rec[lane][i];
+        m = rc.m; S = rc.S; sum_z = rc.sum_z; S_T = rc.S_T; seg = rc.seg;
       }
+      cl_warp_combine<T>(m, seg, S, sum_z, S_T, !t_one || i == N, inv_T);
       ClPart p;
-      p.m = m; p.S = S; p.sum_z = sum_z; p.S_T = S_T; p.col = 0x7fffffff; p.zy = 0.f; p.has_y = 0; p.pad = 0;
-      if (tid < N) {
-        const T* sl = reinterpret_cast<const T*>(slices + (size_t)tid * a.slice_bytes);
+      p.m = m; p.S = S; p.sum_z = sum_z; p.S_T = S_T; p.col = 0x7fffffff; p.zy = 0.f;
+      if (i < N) {
+        const T* sl = reinterpret_cast<const T*>(slices + (size_t)i * a.slice_bytes);
         if (seg >= seg_begin && seg < seg_end) {   // first column of that segment that attains the maximum
 #pragma unroll
           for (int e = V - 1; e >= 0; --e) {
@@ -443,28 +554,22 @@ __global__ void __launch_bounds__(kClThreads, 2) rows_cluster_kernel(const __gri
         const int seg_y = (g.head + y) / V;
         if (seg_y >= seg_begin && seg_y < seg_end) {
           p.zy = Elem<T>::to_f32(sl[(size_t)(seg_y - seg_begin) * V + (g.head + y) % V]);
-          p.has_y = 1;
         }
       }
-      ctrl->part[par][tid] = p;
+      if (lane < K) *cluster.map_shared_rank(&ctrl->gather[par][rank][i], lane) = p;
     }
-    cluster.sync();   // every CTA's partial results of this row are written (and its work on the previous row is done)
+    cluster.sync();   // every CTA's partial results of this row have arrived (and its work on the previous row is done)
 
     // ================= statistics of the whole row: warp i combines the K partial results of tensor i
     for (int i = warp; i < NSTAT; i += NW) {
       ClPart p;
-      p.m = -3.0e38f; p.col = 0x7fffffff; p.S = 0.f; p.sum_z = 0.f; p.S_T = 0.f; p.zy = 0.f; p.has_y = 0; p.pad = 0;
-      if (lane < K) p = *cluster.map_shared_rank(&ctrl->part[par][i], lane);
-      const unsigned key = float_order_key(p.m + 0.f);
-      const unsigned key_m = __reduce_max_sync(0xffffffffu, key);
-      const float m = float_from_order_key(key_m);
+      p.m = -3.0e38f; p.col = 0x7fffffff; p.S = 0.f; p.sum_z = 0.f; p.S_T = 0.f; p.zy = 0.f;
+      if (lane < K) p = ctrl->gather[par][lane][i];
       ClStat st;
-      st.m = m;
-      st.col = (int)__reduce_min_sync(0xffffffffu, key == key_m ? (unsigned)p.col : 0x7fffffffu);
-      st.S = warp_sum(p.S * rescale_exp2<T>((p.m - m) * kLog2e));
-      st.S_T = (t_one && i < N) ? st.S : warp_sum(p.S_T * rescale_exp2<T>((p.m - m) * (kLog2e * inv_T)));
-      st.sum_z = warp_sum(p.sum_z);
-      st.zy = warp_sum(p.has_y ? p.zy : 0.f);
+      st.m = p.m; st.col = p.col; st.S = p.S; st.sum_z = p.sum_z; st.S_T = p.S_T;
+      cl_warp_combine<T>(st.m, st.col, st.S, st.sum_z, st.S_T, !t_one || i == N, inv_T);
+      if (t_one && i < N) st.S_T = st.S;
+      st.zy = warp_sum(p.zy);
       if (lane == 0) ctrl->stat[i] = st;
     }
     if (rank == 0 && v >= 1) finish_row(par ^ 1);   // the previous valid row: all its distance partials are in
@@ -473,94 +578,26 @@ __global__ void __launch_bounds__(kClThreads, 2) rows_cluster_kernel(const __gri
       ctrl->pend[par][tid] = ctrl->stat[tid];
       if (tid == 0) { ctrl->pend_row[par] = r; ctrl->pend_y[par] = y; }
     }
-    float mi[N], cpi[N], cmi[N];                       // per model: maximum, w / S, class mean removed before the distance
-    float cti[KL ? NSTAT : 1], lsi[KL ? NSTAT : 1];    // KL: 1 / S_T and log S_T
+    float class_mean_avg = 0.f;
+#pragma unroll
+    for (int i = 0; i < N; ++i) class_mean_avg += ctrl->stat[i].sum_z;
+    class_mean_avg *= inv_C / (float)N;
 #pragma unroll
     for (int i = 0; i < N; ++i) {
       const ClStat st = ctrl->stat[i];
-      mi[i] = st.m;
-      cpi[i] = w * __frcp_rn(st.S);
-      cmi[i] = a.centred ? st.sum_z * inv_C : 0.f;
-      if constexpr (KL) { cti[i] = __frcp_rn(st.S_T); lsi[i] = logf(st.S_T); }
+      cx.mi[i] = st.m;
+      cx.cpi[i] = w * __frcp_rn(st.S);
+      cx.cmi[i] = class_mean_avg - st.sum_z * inv_C;
+      if constexpr (KL) { cx.cti[i] = __frcp_rn(st.S_T); cx.lsi[i] = logf(st.S_T); }
     }
-    float mb = 0.f;   // KL mean target: maximum of the averaged peers
-    if constexpr (KLM) { const ClStat st = ctrl->stat[N]; mb = st.m; cti[N] = __frcp_rn(st.S_T); lsi[N] = logf(st.S_T); }
+    if constexpr (KLM) { const ClStat st = ctrl->stat[N]; cx.mb = st.m; cx.cti[N] = __frcp_rn(st.S_T); cx.lsi[N] = logf(st.S_T); }
+    cx.y = y;
 
     // ================= pass B: distance terms and gradients, the n models side by side
-    float2 dist2[NOUT], qs2 = make_float2(0.f, 0.f);
+    ClColAcc<NOUT> acc;
+    acc.qs2 = make_float2(0.f, 0.f);
 #pragma unroll
-    for (int i = 0; i < NOUT; ++i) dist2[i] = make_float2(0.f, 0.f);
-    // Two neighbouring columns c, c + 1 (first_in / second_in: inside the row); zc: the n models' logits.
-    // Returns the gradient pairs of the requested models; `lab` says that c or c + 1 may be the label column.
-    auto column2 = [&](bool ragged, const float2 (&zc)[N], float2 (&gc)[NOUT], int64_t c, bool lab, bool first_in, bool second_in) {
-      const bool kRagged = ragged;   // some column of the pair may lie outside the row
-      float2 ncq = make_float2(-cq, -cq);
-      if (lab) ncq = make_float2((c == (int64_t)y) ? -(cq + cy) : -cq, (c + 1 == (int64_t)y) ? -(cq + cy) : -cq);
-      const float2 in2 = make_float2(first_in ? 1.f : 0.f, second_in ? 1.f : 0.f);
-      auto inside = [&](float2 x) { return kRagged ? __fmul2_rn(x, in2) : x; };
-      if constexpr (MODE == kClMse) {
-        float2 zp[N], mu = make_float2(0.f, 0.f), q = make_float2(0.f, 0.f);
-#pragma unroll
-        for (int i = 0; i < N; ++i) { zp[i] = __fadd2_rn(zc[i], make_float2(-cmi[i], -cmi[i])); mu = __fadd2_rn(mu, zp[i]); }
-        mu = __fmul2_rn(mu, make_float2(-1.f / (float)N, -1.f / (float)N));
-#pragma unroll
-        for (int i = 0; i < N; ++i) {
-          zp[i] = inside(__fadd2_rn(zp[i], mu));
-          q = __ffma2_rn(zp[i], zp[i], q);
-        }
-#pragma unroll
-        for (int i = 0; i < NOUT; ++i) {
-          const float nm = -mi[i] * kLog2e;
-          const float2 e = exp_shift2<T>(zc[i], mi[i], make_float2(kLog2e, kLog2e), make_float2(nm, nm));
-          gc[i] = __ffma2_rn(e, make_float2(cpi[i], cpi[i]), __ffma2_rn(make_float2(cd, cd), zp[i], ncq));
-          dist2[i] = __ffma2_rn(zp[i], zp[i], dist2[i]);
-        }
-        qs2 = __fadd2_rn(qs2, q);
-      } else if constexpr (MODE == kClKlPairwise) {
-        float2 t[N], lt[N], Q = make_float2(0.f, 0.f), E = make_float2(0.f, 0.f);
-#pragma unroll
-        for (int i = 0; i < N; ++i) {
-          float2 e1 = make_float2(0.f, 0.f), et;
-          if (t_one || i < NOUT) {
-            const float nm = -mi[i] * kLog2e;
-            e1 = exp_shift2<T>(zc[i], mi[i], make_float2(kLog2e, kLog2e), make_float2(nm, nm));
-          }
-          et = t_one ? e1 : exp_temp2<T>(zc[i], mi[i], inv_T, kLog2e * inv_T);
-          t[i] = inside(__fmul2_rn(et, make_float2(cti[i], cti[i])));
-          const float2 x = __fadd2_rn(zc[i], make_float2(-mi[i], -mi[i]));
-          const float2 l = __ffma2_rn(x, make_float2(inv_T, inv_T), make_float2(-lsi[i], -lsi[i]));
-          lt[i] = make_float2(fmaxf(l.x, -3.0e38f), fmaxf(l.y, -3.0e38f));   // log t_i, kept finite: 0 * log 0 = 0
-          Q = __fadd2_rn(Q, t[i]);
-          E = __ffma2_rn(t[i], lt[i], E);
-          if (i < NOUT) gc[i] = __ffma2_rn(e1, make_float2(cpi[i], cpi[i]), ncq);
-        }
-        const float2 nQ = make_float2(-Q.x, -Q.y);
-#pragma unroll
-        for (int i = 0; i < NOUT; ++i) {
-          gc[i] = __ffma2_rn(make_float2(ckl, ckl), __ffma2_rn(make_float2((float)N, (float)N), t[i], nQ), gc[i]);
-          dist2[i] = __fadd2_rn(dist2[i], __ffma2_rn(nQ, lt[i], E));   // sum_{j != i} t_j (log t_j - log t_i)
-        }
-      } else {
-        // KL to the softmax of the averaged peers: t = softmax(zbar / T), p^T = softmax(z_0 / T)
-        const float inv_P = 1.f / (float)(N - 1);
-        float2 zb = make_float2(0.f, 0.f);
-#pragma unroll
-        for (int j = 1; j < N; ++j) zb = __fadd2_rn(zb, zc[j]);
-        zb = __fmul2_rn(zb, make_float2(inv_P, inv_P));
-        const float nm = -mi[0] * kLog2e;
-        const float2 e1 = exp_shift2<T>(zc[0], mi[0], make_float2(kLog2e, kLog2e), make_float2(nm, nm));
-        const float2 eT = t_one ? e1 : exp_temp2<T>(zc[0], mi[0], inv_T, kLog2e * inv_T);
-        const float2 pT = __fmul2_rn(eT, make_float2(cti[0], cti[0]));
-        const float2 x0 = __fadd2_rn(zc[0], make_float2(-mi[0], -mi[0]));
-        const float2 lp = __ffma2_rn(x0, make_float2(inv_T, inv_T), make_float2(-lsi[0], -lsi[0]));
-        const float2 tb = inside(__fmul2_rn(exp_temp2<T>(zb, mb, inv_T, kLog2e * inv_T), make_float2(cti[N], cti[N])));
-        const float2 xb = __fadd2_rn(zb, make_float2(-mb, -mb));
-        const float2 lb = __ffma2_rn(xb, make_float2(inv_T, inv_T), make_float2(-lsi[N], -lsi[N]));
-        const float2 dl = make_float2(fmaxf(lb.x, -3.0e38f) - fmaxf(lp.x, -3.0e38f), fmaxf(lb.y, -3.0e38f) - fmaxf(lp.y, -3.0e38f));
-        gc[0] = __ffma2_rn(make_float2(ckl, ckl), __fadd2_rn(pT, make_float2(-tb.x, -tb.y)), __ffma2_rn(e1, make_float2(cpi[0], cpi[0]), ncq));
-        dist2[0] = __ffma2_rn(tb, dl, dist2[0]);
-      }
-    };
+    for (int i = 0; i < NOUT; ++i) acc.dist2[i] = make_float2(0.f, 0.f);
     const int seg_y = (g.head + y) / V;
     for (int q = tid; q < nseg; q += NT) {
       const int s = seg_begin + q;
@@ -583,7 +620,7 @@ __global__ void __launch_bounds__(kClThreads, 2) rows_cluster_kernel(const __gri
               zc[i] = make_float2(__uint_as_float(word << 16), __uint_as_float(word & 0xFFFF0000u));
             }
           }
-          column2(false, zc, gc, cbase + 2 * h, lab, true, true);
+          cl_column2<T, N, MODE, ALL, false>(cx, acc, zc, gc, cbase + 2 * h, lab, make_float2(1.f, 1.f));
 #pragma unroll
           for (int i = 0; i < NOUT; ++i) {
             if constexpr (ES == 4) {
@@ -609,9 +646,9 @@ __global__ void __launch_bounds__(kClThreads, 2) rows_cluster_kernel(const __gri
 #pragma unroll
           for (int i = 0; i < N; ++i) {
             const T* el = reinterpret_cast<const T*>(slices + (size_t)i * a.slice_bytes + (size_t)q * 16) + 2 * h;
-            zc[i] = make_float2(in0 ? Elem<T>::to_f32(el[0]) : mi[i], in1 ? Elem<T>::to_f32(el[1]) : mi[i]);
+            zc[i] = make_float2(in0 ? Elem<T>::to_f32(el[0]) : cx.mi[i], in1 ? Elem<T>::to_f32(el[1]) : cx.mi[i]);
           }
-          column2(true, zc, gc, c0, lab, in0, in1);
+          cl_column2<T, N, MODE, ALL, true>(cx, acc, zc, gc, c0, lab, make_float2(in0 ? 1.f : 0.f, in1 ? 1.f : 0.f));
 #pragma unroll
           for (int i = 0; i < NOUT; ++i) {
             if (a.grad[i] == nullptr) continue;
@@ -623,14 +660,19 @@ __global__ void __launch_bounds__(kClThreads, 2) rows_cluster_kernel(const __gri
       }
     }
 
-    // ================= distance partial sums of this CTA (read by CTA 0 behind the next cluster barrier)
+    // ================= distance partial sums of this CTA, handed to CTA 0 (which reads them behind the next cluster barrier)
 #pragma unroll
     for (int i = 0; i < NOUT; ++i) {
-      const float dw = warp_sum(dist2[i].x + dist2[i].y);
+      const float dw = warp_sum(acc.dist2[i].x + acc.dist2[i].y);
       if (lane == 0) ctrl->dwarp[warp][i] = dw;
     }
     if constexpr (MODE == kClMse) {
-      const float qw = warp_sum(qs2.x + qs2.y);
+      float qt = acc.qs2.x + acc.qs2.y;
+      if constexpr (ALL) {
+#pragma unroll
+        for (int i = 0; i < N; ++i) qt += acc.dist2[i].x + acc.dist2[i].y;
+      }
+      const float qw = warp_sum(qt);
       if (lane == 0) ctrl->dwarp[warp][kClMax] = qw;
     }
     __syncthreads();   // pass B has read the ranges: they may be overwritten; the warps' partial sums are in place
@@ -640,25 +682,26 @@ __global__ void __launch_bounds__(kClThreads, 2) rows_cluster_kernel(const __gri
       while (r2 < a.row_end && !row_is_valid(r2)) r2 += ncl;
       if (r2 < a.row_end) { issue_row(r2); issued = r2; }
     }
-    if (tid <= kClMax && (tid < NOUT || tid == kClMax)) {
+    if (tid >= 32 && tid - 32 <= kClMax && (tid - 32 < NOUT || tid - 32 == kClMax)) {
+      const int i = tid - 32;
       float d = 0.f;
-      if (tid < NOUT || MODE == kClMse) {
+      if (i < NOUT || MODE == kClMse) {
 #pragma unroll
-        for (int wv = 0; wv < NW; ++wv) d += ctrl->dwarp[wv][tid];
+        for (int wv = 0; wv < NW; ++wv) d += ctrl->dwarp[wv][i];
       }
-      ctrl->dpart[par][tid] = d;
+      *cluster.map_shared_rank(&ctrl->dgather[par][rank][i], 0) = d;
     }
     ++v;
   }
 
-  // ---------------- the last valid row's loss; nobody leaves while its shared memory may still be read
+  // ---------------- the last valid row's loss; nobody leaves while its shared memory may still be written
   cluster.sync();
   if (rank == 0 && v >= 1) finish_row((v - 1) & 1);
   if (ctrl->abort_flag && tid == 0) {
     // a wait ran out: give copies that may still be in flight one more bounded interval before the CTA ends
-    mbar_wait_limited(&ctrl->full, (uint32_t)(v + 1) & 1u, &ctrl->abort_flag, &a.hdr->status, CODISTILL_DEV_TIMEOUT, kClDrainLimitNs, false, true);
+    for (int i = 0; i < N; ++i)
+      mbar_wait_limited(&ctrl->full[i], (uint32_t)(v + 1) & 1u, &ctrl->abort_flag, &a.hdr->status, CODISTILL_DEV_TIMEOUT, kClDrainLimitNs, false, true);
   }
-  cluster.sync();
 }
 
 // ------------------------------------------------------------------ host side
@@ -743,6 +786,9 @@ static cudaError_t cluster_launch_one(const ClArgs& a, const ClPlan& p, cudaStre
       if ((e = cuda_note(cudaOccupancyMaxActiveClusters(&max_clusters, kernel, &cfg), "cudaOccupancyMaxActiveClusters")) != cudaSuccess) return e;
       if (max_clusters < 1) return cuda_note(cudaErrorLaunchOutOfResources, "no cluster of this size fits the device");
       known[key] = max_clusters;
+      if (getenv("CODISTILL_VERBOSE"))
+        fprintf(stderr, "codistill: cluster kernel n=%d: %d CTAs per cluster, %u bytes of shared memory per CTA, %d clusters co-resident\n",
+                N, p.cluster, p.smem_bytes, max_clusters);
     }
   }
   const int64_t rows = a.row_end - a.row_begin;
