@@ -110,11 +110,12 @@ def load_library() -> ctypes.CDLL:
     global _lib
     if _lib is not None:
         return _lib
-    if not os.path.exists(LIB_PATH):
+    path = os.environ.get("CODISTILL_LIBRARY", LIB_PATH)   # another build of the same library (same ABI), e.g. for A/B timing
+    if not os.path.exists(path):
         raise RuntimeError(
-            f"{LIB_PATH} is missing: build it with `python -m paper_2010_02838_b200.build` "
+            f"{path} is missing: build it with `python -m paper_2010_02838_b200.build` "
             "(nvcc, sm_100a). There is no CPU or PyTorch fallback for the codistillation kernels.")
-    lib = ctypes.CDLL(LIB_PATH)
+    lib = ctypes.CDLL(path)
     vp, i64, i32, f32 = ctypes.c_void_p, ctypes.c_int64, ctypes.c_int, ctypes.c_float
     lib.codistill_loss_fwd_bwd.restype = i32
     lib.codistill_loss_fwd_bwd.argtypes = [vp, ctypes.POINTER(vp), vp, vp, i32, i64, i64, f32, f32, i32, vp, vp, vp, vp]

@@ -173,9 +173,6 @@ static Regime pick_regime(const KArgs& a, int dtype, int smem_optin) {
     if (strcmp(want, "cluster") == 0 && can_cluster) return kRegimeCluster;
     if (strcmp(want, "block") == 0) return generic;
   }
-  // Distances whose gradient needs row statistics of the peers (softmax-KL, centred MSE) would read the
-  // peers twice from global memory: the cluster-resident kernel keeps all n rows on chip instead.
-  if (can_cluster && a.dist != CODISTILL_DIST_MSE_LOGITS) return kRegimeCluster;
   if (can_tma && (!can_stream || tma_ctas_per_sm(a, dtype, smem_optin) >= 2)) return kRegimeTma;
   if (can_stream) return kRegimeStream;
   if (can_cluster) return kRegimeCluster;   // peer counts the two MSE kernels above are not built for (4, 5, 6)

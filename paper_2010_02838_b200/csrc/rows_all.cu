@@ -671,13 +671,14 @@ extern "C" int codistill_loss_fwd_bwd_all(const codistill_all_params_t* p, void*
 
   if (const int rc_cuda = cuda_status(launch_prep_rows(a.hdr, const_cast<int64_t*>(a.partials), a.labels, a.mask, a.rows, a.classes, stream))) return rc_cuda;
   if (a.rows > 0) {
-    // Long rows: the cluster-resident kernel reads every logit from HBM once (the n row images of a row
-    // index stay in the shared memory of a cluster); the direct-load kernel above reads them twice.
-    // CODISTILL_REGIME=stream keeps the direct-load kernel (for measurements).
+    // On request (CODISTILL_REGIME=cluster) long rows go to the cluster-resident kernel, which reads every
+    // logit from HBM once (the n row images of a row index stay in the shared memory of a cluster) where the
+    // direct-load kernel above reads them twice; it is the slower of the two at present (bound by instruction
+    // issue, not by memory), so it is not the default.
     const char* want = getenv("CODISTILL_REGIME");
-    const bool keep_direct = want != nullptr && strcmp(want, "stream") == 0;
+    const bool use_cluster = want != nullptr && strcmp(want, "cluster") == 0;
     cudaError_t e;
-    if (!keep_direct && cluster_fits(p->n, p->classes, p->row_stride, p->dtype, smem_optin)) {
+    if (use_cluster && cluster_fits(p->n, p->classes, p->row_stride, p->dtype, smem_optin)) {
       ClArgs c;
       memset(&c, 0, sizeof(c));
       for (int i = 0; i < p->n; ++i) { c.model[i] = a.model[i]; c.grad[i] = a.grad[i]; }

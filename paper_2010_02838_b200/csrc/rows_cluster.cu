@@ -95,61 +95,80 @@ __device__ __forceinline__ float exp_nat1(float x) {
   if constexpr (sizeof(T) == 4) return expf(x); else return ex2_approx(x * kLog2e);
 }
 
-// Running statistics of one thread over its segments of one tensor (visited in rising order); one
-// partial sum per pair position of a segment, so that the additions of a segment do not form a chain.
-template <int H>
-struct ClAcc {
-  float best;       // finite start value, so that the first rescale is exp2(-huge) = 0 and never NaN
-  int best_seg;
-  float2 s2[H], t2[H], zs2[H];
-  __device__ __forceinline__ void reset() {
-    best = -3.0e38f;
-    best_seg = 0x7fffffff;
-#pragma unroll
-    for (int h = 0; h < H; ++h) { s2[h] = make_float2(0.f, 0.f); t2[h] = s2[h]; zs2[h] = s2[h]; }
-  }
-};
+// One lane's statistics of its segments of one tensor; the sums are relative to `best`.
+struct ClLane { float best; int seg; float s, z, t; };
 
-template <typename T, bool TEMP, int H>
-__device__ __forceinline__ void cl_raise(ClAcc<H>& acc, float fm, int s, float inv_T) {
-  if (fm > acc.best) {
-    const float sc = rescale_exp2<T>((acc.best - fm) * kLog2e);
-#pragma unroll
-    for (int h = 0; h < H; ++h) acc.s2[h] = __fmul2_rn(acc.s2[h], make_float2(sc, sc));
-    if constexpr (TEMP) {
-      const float st = rescale_exp2<T>((acc.best - fm) * (kLog2e * inv_T));
-#pragma unroll
-      for (int h = 0; h < H; ++h) acc.t2[h] = __fmul2_rn(acc.t2[h], make_float2(st, st));
-    }
-    acc.best = fm;
-    acc.best_seg = s;
-  }
-}
-
-// one whole segment (all of its columns lie inside the row)
+// Statistics of the lane's share of segments [q_lo, q_hi) of one tensor's range (all of them whole segments
+// inside the row), four segments at a time: the maximum of the batch first, then the exponentials against a
+// fixed reference -- no branch in the loop body.  Lanes without a segment return best = -3e38, sums 0.
 template <typename T, bool TEMP>
-__device__ __forceinline__ void cl_sweep_seg(ClAcc<SegOps<T>::H>& acc, const uint4& raw, int s, float inv_T, bool need_z) {
+__device__ __forceinline__ ClLane cl_sweep_range(const char* sl, int q_lo, int q_hi, int seg_begin, int tid, float inv_T, bool need_z) {
   constexpr int H = SegOps<T>::H;
-  cl_raise<T, TEMP>(acc, SegOps<T>::to_float(SegOps<T>::fold(raw)), s, inv_T);
+  constexpr int U = 4;
+  constexpr uint32_t kPad = sizeof(T) == 4 ? 0xFF800000u : 0xFF80FF80u;   // -inf in every element: no maximum, exp = 0
+  ClLane L;
+  L.best = -3.0e38f; L.seg = 0x7fffffff; L.s = 0.f; L.z = 0.f; L.t = 0.f;
+  float2 s2[H], t2[H], zs2[H];
+#pragma unroll
+  for (int h = 0; h < H; ++h) { s2[h] = make_float2(0.f, 0.f); t2[h] = s2[h]; zs2[h] = s2[h]; }
   const float2 l2e2 = make_float2(kLog2e, kLog2e);
-  const float2 nmk = make_float2(-acc.best * kLog2e, -acc.best * kLog2e);
-  float2 z2[H];
-  SegOps<T>::unpack2(raw, z2);
+#pragma unroll 1
+  for (int q = q_lo + tid; q < q_hi; q += U * kClThreads) {
+    uint4 raw[U];
+    float fm[U];
+    bool ok[U];
 #pragma unroll
-  for (int h = 0; h < H; ++h) {
-    acc.s2[h] = __fadd2_rn(acc.s2[h], exp_shift2<T>(z2[h], acc.best, l2e2, nmk));
-    if constexpr (TEMP) acc.t2[h] = __fadd2_rn(acc.t2[h], exp_temp2<T>(z2[h], acc.best, inv_T, kLog2e * inv_T));
-  }
-  if (need_z) {   // the sum of the logits: label smoothing and the centred distance only
+    for (int u = 0; u < U; ++u) {
+      const int qq = q + u * kClThreads;
+      ok[u] = qq < q_hi;
+      raw[u] = ok[u] ? *reinterpret_cast<const uint4*>(sl + (size_t)qq * 16) : make_uint4(kPad, kPad, kPad, kPad);
+      fm[u] = SegOps<T>::to_float(SegOps<T>::fold(raw[u]));
+    }
+    const float bm = fmaxf(fmaxf(fm[0], fm[1]), fmaxf(fm[2], fm[3]));
+    int sb = seg_begin + q + (U - 1) * kClThreads;   // the first segment of the batch that attains its maximum
 #pragma unroll
-    for (int h = 0; h < H; ++h) acc.zs2[h] = __fadd2_rn(acc.zs2[h], z2[h]);
+    for (int u = U - 2; u >= 0; --u) sb = fm[u] == bm ? seg_begin + q + u * kClThreads : sb;
+    const float nb = fmaxf(L.best, bm);
+    const float sc = rescale_exp2<T>((L.best - nb) * kLog2e);
+#pragma unroll
+    for (int h = 0; h < H; ++h) s2[h] = __fmul2_rn(s2[h], make_float2(sc, sc));
+    if constexpr (TEMP) {
+      const float st = rescale_exp2<T>((L.best - nb) * (kLog2e * inv_T));
+#pragma unroll
+      for (int h = 0; h < H; ++h) t2[h] = __fmul2_rn(t2[h], make_float2(st, st));
+    }
+    L.seg = bm > L.best ? sb : L.seg;
+    L.best = nb;
+    const float2 nmk = make_float2(-nb * kLog2e, -nb * kLog2e);
+#pragma unroll
+    for (int u = 0; u < U; ++u) {
+      if (u > 0 && !ok[u]) continue;   // padding: nothing to add (the same for all lanes of most warps)
+      float2 z2[H];
+      SegOps<T>::unpack2(raw[u], z2);
+#pragma unroll
+      for (int h = 0; h < H; ++h) {
+        s2[h] = __fadd2_rn(s2[h], exp_shift2<T>(z2[h], nb, l2e2, nmk));
+        if constexpr (TEMP) t2[h] = __fadd2_rn(t2[h], exp_temp2<T>(z2[h], nb, inv_T, kLog2e * inv_T));
+      }
+      if (need_z) {   // the sum of the logits: label smoothing and the centred distance only
+#pragma unroll
+        for (int h = 0; h < H; ++h) zs2[h] = __fadd2_rn(zs2[h], z2[h]);
+      }
+    }
   }
+  float2 sa = s2[0], ta = t2[0], za = zs2[0];
+#pragma unroll
+  for (int h = 1; h < H; ++h) { sa = __fadd2_rn(sa, s2[h]); ta = __fadd2_rn(ta, t2[h]); za = __fadd2_rn(za, zs2[h]); }
+  L.s = sa.x + sa.y;
+  L.t = ta.x + ta.y;
+  L.z = za.x + za.y;
+  return L;
 }
 
-// a ragged segment (first or last of the row image): only the columns inside the row count
-// (accumulators in and out by value, so that the caller's copy stays in registers)
+// Adds one ragged segment (first or last of the row image: only the columns inside the row count) to a
+// lane's statistics.  In and out by value, so that the caller's copy stays in registers.
 template <typename T, bool TEMP>
-__device__ __noinline__ ClAcc<SegOps<T>::H> cl_sweep_edge(ClAcc<SegOps<T>::H> acc, uint4 raw, int s, int head, int64_t C, float inv_T) {
+__device__ __noinline__ ClLane cl_sweep_edge(ClLane L, uint4 raw, int s, int head, int64_t C, float inv_T) {
   constexpr int V = SegOps<T>::V;
   float z[V];
   SegOps<T>::unpack(raw, z);
@@ -159,39 +178,50 @@ __device__ __noinline__ ClAcc<SegOps<T>::H> cl_sweep_edge(ClAcc<SegOps<T>::H> ac
     const int64_t c = (int64_t)s * V - head + e;
     if (c >= 0 && c < C) fm = fmaxf(fm, z[e]);
   }
-  cl_raise<T, TEMP>(acc, fm, s, inv_T);
+  // the ragged segments are the first or the last of the row: an equal maximum in segment 0 comes first
+  const bool take = fm > L.best || (fm == L.best && s < L.seg);
+  const float nb = fmaxf(L.best, fm);
+  L.s *= rescale_exp2<T>((L.best - nb) * kLog2e);
+  if constexpr (TEMP) L.t *= rescale_exp2<T>((L.best - nb) * (kLog2e * inv_T));
+  if (take) L.seg = s;
+  L.best = nb;
   const float2 l2e2 = make_float2(kLog2e, kLog2e);
-  const float2 nmk = make_float2(-acc.best * kLog2e, -acc.best * kLog2e);
+  const float2 nmk = make_float2(-nb * kLog2e, -nb * kLog2e);
 #pragma unroll
   for (int e = 0; e < V; ++e) {
     const int64_t c = (int64_t)s * V - head + e;
     if (c >= 0 && c < C) {
-      acc.s2[0].x += exp_shift2<T>(make_float2(z[e], z[e]), acc.best, l2e2, nmk).x;
-      acc.zs2[0].x += z[e];
-      if constexpr (TEMP) acc.t2[0].x += exp_temp2<T>(make_float2(z[e], z[e]), acc.best, inv_T, kLog2e * inv_T).x;
+      L.s += exp_shift2<T>(make_float2(z[e], z[e]), nb, l2e2, nmk).x;
+      L.z += z[e];
+      if constexpr (TEMP) L.t += exp_temp2<T>(make_float2(z[e], z[e]), nb, inv_T, kLog2e * inv_T).x;
     }
   }
-  return acc;
+  return L;
 }
 
-// Reduces the lanes' accumulators of one sub-range to one record (all lanes take part).
-template <typename T, bool TEMP, int H>
-__device__ __forceinline__ ClRec cl_warp_record(const ClAcc<H>& acc, int tensor, float inv_T) {
-  const unsigned key = float_order_key(acc.best + 0.f);   // -0 is folded onto +0: they tie
-  const unsigned key_w = __reduce_max_sync(0xffffffffu, key);
-  float s_t = 0.f, z_t = 0.f, t_t = 0.f;
+// Sums NV per-lane values (NV a power of two, 2..32) across the warp in NV - 1 + log2(32 / NV) shuffles instead of
+// 5 NV: in each step a lane hands one half of its values to its partner and keeps the other half.  On
+// return v[0] of lane L is the total of value number L >> (5 - log2 NV).
+template <int NV>
+__device__ __forceinline__ void warp_multi_sum(float (&v)[NV], int lane) {
+  static_assert(NV >= 2 && NV <= 32 && (NV & (NV - 1)) == 0, "a power of two");
+  int off = 16;
 #pragma unroll
-  for (int h = 0; h < H; ++h) { s_t += acc.s2[h].x + acc.s2[h].y; z_t += acc.zs2[h].x + acc.zs2[h].y; t_t += acc.t2[h].x + acc.t2[h].y; }
-  ClRec r;
-  r.seg = (int)__reduce_min_sync(0xffffffffu, key == key_w ? (unsigned)acc.best_seg : 0x7fffffffu);
-  r.m = float_from_order_key(key_w);
-  r.S = warp_sum(s_t * rescale_exp2<T>((acc.best - r.m) * kLog2e));
-  r.sum_z = warp_sum(z_t);
-  r.S_T = 0.f;
-  if constexpr (TEMP) r.S_T = warp_sum(t_t * rescale_exp2<T>((acc.best - r.m) * (kLog2e * inv_T)));
-  r.tensor = tensor;
-  return r;
+  for (int cnt = NV; cnt > 1; cnt >>= 1, off >>= 1) {
+    const int half = cnt >> 1;
+    const bool upper = (lane & off) != 0;
+#pragma unroll
+    for (int k = 0; k < half; ++k) {
+      const float send = upper ? v[k] : v[k + half];
+      const float keep = upper ? v[k + half] : v[k];
+      v[k] = keep + __shfl_xor_sync(0xffffffffu, send, off);
+    }
+  }
+#pragma unroll
+  for (; off > 0; off >>= 1) v[0] += __shfl_xor_sync(0xffffffffu, v[0], off);
 }
+__host__ __device__ constexpr int cl_pow2_at_least(int x) { return x <= 2 ? 2 : x <= 4 ? 4 : x <= 8 ? 8 : x <= 16 ? 16 : 32; }
+__host__ __device__ constexpr int cl_log2(int x) { return x <= 2 ? 1 : x <= 4 ? 2 : x <= 8 ? 3 : x <= 16 ? 4 : 5; }
 
 // Combines partial results (one per lane; lanes without one pass m = -3e38, S = 0, pos = INT_MAX) across
 // the warp: the maximum, the lowest position among those that attain it, the sums rescaled to it.
@@ -210,32 +240,44 @@ __device__ __forceinline__ void cl_warp_combine(float& m, int& pos, float& S, fl
 // What pass B needs of the row statistics (registers), and its running sums.
 template <int N, int NS>
 struct ClColCtx {
-  float mi[N], cpi[N], cmi[N];   // per model: maximum, w / S, centred distance: -(class mean - average class mean of the models)
+  float nml[N], cpi[N];          // per model: -maximum * log2(e) (bf16 logits) or -maximum (fp32 logits), and w / S
   float cti[NS], lsi[NS];        // KL: 1 / S_T and log S_T (slot N: the averaged peers)
   float mb;                      // KL mean target: maximum of the averaged peers
   float cd, cq, cy, ckl, inv_T;
   bool t_one, centred;
   int y;
+  const ClStat* stat;            // shared memory: the full statistics (maxima for the KL logarithms, class means)
+  float cmean;                   // centred distance: average over the models of their class means
+  float inv_C;
 };
 template <int NOUT>
 struct ClColAcc {
   float2 dist2[NOUT], qs2;
 };
 
+// exp(z - m) for a pair of columns from the precomputed -m (see ClColCtx::nml)
+template <typename T>
+__device__ __forceinline__ float2 exp_from_nml(float2 z, float nml) {
+  if constexpr (sizeof(T) == 4) {
+    return make_float2(expf(z.x + nml), expf(z.y + nml));
+  } else {
+    const float2 t = __ffma2_rn(z, make_float2(kLog2e, kLog2e), make_float2(nml, nml));
+    return make_float2(ex2_approx(t.x), ex2_approx(t.y));
+  }
+}
+
 // Two neighbouring columns c, c + 1 of the n models (zc): distance terms into `acc`, gradient pairs of the
-// requested models into gc.  `lab`: c or c + 1 may be the label column.  RAGGED: a column of the pair may lie
-// outside the row (in2 = 1 / 0 per column); such columns contribute nothing.
-template <typename T, int N, int MODE, bool ALL, bool RAGGED, int NS>
+// requested models into gc.  LAB: c or c + 1 may be the label column.  MASKED: the distance terms of the two
+// columns count with the weights in2 (1 / 0: a column outside the row, or a column done before, adds nothing).
+template <typename T, int N, int MODE, bool ALL, bool LAB, bool MASKED, int NS>
 __device__ __forceinline__ void cl_column2(const ClColCtx<N, NS>& x, ClColAcc<ALL ? N : 1>& acc, const float2 (&zc)[N],
-                                           float2 (&gc)[ALL ? N : 1], int64_t c, bool lab, float2 in2) {
+                                           float2 (&gc)[ALL ? N : 1], int64_t c, float2 in2) {
   constexpr int NOUT = ALL ? N : 1;
   float2 ncq = make_float2(-x.cq, -x.cq);
-  if (lab) ncq = make_float2((c == (int64_t)x.y) ? -(x.cq + x.cy) : -x.cq, (c + 1 == (int64_t)x.y) ? -(x.cq + x.cy) : -x.cq);
-  auto inside = [&](float2 v) { if constexpr (RAGGED) return __fmul2_rn(v, in2); else return v; };
-  const float2 l2e2 = make_float2(kLog2e, kLog2e);
+  if constexpr (LAB) ncq = make_float2((c == (int64_t)x.y) ? -(x.cq + x.cy) : -x.cq, (c + 1 == (int64_t)x.y) ? -(x.cq + x.cy) : -x.cq);
+  auto counted = [&](float2 v) { if constexpr (MASKED) return __fmul2_rn(v, in2); else return v; };
   if constexpr (MODE == kClMse) {
-    // z'_i = z_i - mean_j z_j, for the centred distance on z_i - (class mean of model i); x.cmi[i] holds
-    // -(class mean_i - mean_j class mean_j), so one addition per model centres both ways
+    // z'_i = z_i - mean_j z_j; for the centred distance z_i loses the class mean of model i first
     float2 zp[N], mu = zc[0];
 #pragma unroll
     for (int i = 1; i < N; ++i) mu = __fadd2_rn(mu, zc[i]);
@@ -244,37 +286,33 @@ __device__ __forceinline__ void cl_column2(const ClColCtx<N, NS>& x, ClColAcc<AL
     for (int i = 0; i < N; ++i) zp[i] = __fadd2_rn(zc[i], mu);
     if (x.centred) {
 #pragma unroll
-      for (int i = 0; i < N; ++i) zp[i] = __fadd2_rn(zp[i], make_float2(x.cmi[i], x.cmi[i]));
-    }
-    if constexpr (RAGGED) {
-#pragma unroll
-      for (int i = 0; i < N; ++i) zp[i] = __fmul2_rn(zp[i], in2);
+      for (int i = 0; i < N; ++i) {
+        const float d = x.cmean - x.stat[i].sum_z * x.inv_C;
+        zp[i] = __fadd2_rn(zp[i], make_float2(d, d));
+      }
     }
     if constexpr (!ALL) {   // sum_j z'_j^2 of the pairwise form (with every model's output it is the sum of their distance sums)
       float2 q = make_float2(0.f, 0.f);
 #pragma unroll
       for (int i = 0; i < N; ++i) q = __ffma2_rn(zp[i], zp[i], q);
-      acc.qs2 = __fadd2_rn(acc.qs2, q);
+      acc.qs2 = __fadd2_rn(acc.qs2, counted(q));
     }
 #pragma unroll
     for (int i = 0; i < NOUT; ++i) {
-      const float nm = -x.mi[i] * kLog2e;
-      const float2 e = exp_shift2<T>(zc[i], x.mi[i], l2e2, make_float2(nm, nm));
+      const float2 e = exp_from_nml<T>(zc[i], x.nml[i]);
       gc[i] = __ffma2_rn(e, make_float2(x.cpi[i], x.cpi[i]), __ffma2_rn(make_float2(x.cd, x.cd), zp[i], ncq));
-      acc.dist2[i] = __ffma2_rn(zp[i], zp[i], acc.dist2[i]);
+      acc.dist2[i] = __ffma2_rn(counted(zp[i]), zp[i], acc.dist2[i]);
     }
   } else if constexpr (MODE == kClKlPairwise) {
     float2 t[N], lt[N], Q = make_float2(0.f, 0.f), E = make_float2(0.f, 0.f);
 #pragma unroll
     for (int i = 0; i < N; ++i) {
+      const float mi = x.stat[i].m;
       float2 e1 = make_float2(0.f, 0.f);
-      if (x.t_one || i < NOUT) {
-        const float nm = -x.mi[i] * kLog2e;
-        e1 = exp_shift2<T>(zc[i], x.mi[i], l2e2, make_float2(nm, nm));
-      }
-      const float2 et = x.t_one ? e1 : exp_temp2<T>(zc[i], x.mi[i], x.inv_T, kLog2e * x.inv_T);
-      t[i] = inside(__fmul2_rn(et, make_float2(x.cti[i], x.cti[i])));
-      const float2 d = __fadd2_rn(zc[i], make_float2(-x.mi[i], -x.mi[i]));
+      if (x.t_one || i < NOUT) e1 = exp_from_nml<T>(zc[i], x.nml[i]);
+      const float2 et = x.t_one ? e1 : exp_temp2<T>(zc[i], mi, x.inv_T, kLog2e * x.inv_T);
+      t[i] = __fmul2_rn(et, make_float2(x.cti[i], x.cti[i]));
+      const float2 d = __fadd2_rn(zc[i], make_float2(-mi, -mi));
       const float2 l = __ffma2_rn(d, make_float2(x.inv_T, x.inv_T), make_float2(-x.lsi[i], -x.lsi[i]));
       lt[i] = make_float2(fmaxf(l.x, -3.0e38f), fmaxf(l.y, -3.0e38f));   // log t_i, kept finite: 0 * log 0 = 0
       Q = __fadd2_rn(Q, t[i]);
@@ -285,29 +323,64 @@ __device__ __forceinline__ void cl_column2(const ClColCtx<N, NS>& x, ClColAcc<AL
 #pragma unroll
     for (int i = 0; i < NOUT; ++i) {
       gc[i] = __ffma2_rn(make_float2(x.ckl, x.ckl), __ffma2_rn(make_float2((float)N, (float)N), t[i], nQ), gc[i]);
-      acc.dist2[i] = __fadd2_rn(acc.dist2[i], __ffma2_rn(nQ, lt[i], E));   // sum_{j != i} t_j (log t_j - log t_i)
+      acc.dist2[i] = __fadd2_rn(acc.dist2[i], counted(__ffma2_rn(nQ, lt[i], E)));   // sum_{j != i} t_j (log t_j - log t_i)
     }
   } else {
     // KL to the softmax of the averaged peers: t = softmax(zbar / T), p^T = softmax(z_0 / T)
     const float inv_P = 1.f / (float)(N - 1);
-    float2 zb = make_float2(0.f, 0.f);
+    const float m0 = x.stat[0].m;
+    float2 zb = zc[1];
 #pragma unroll
-    for (int j = 1; j < N; ++j) zb = __fadd2_rn(zb, zc[j]);
+    for (int j = 2; j < N; ++j) zb = __fadd2_rn(zb, zc[j]);
     zb = __fmul2_rn(zb, make_float2(inv_P, inv_P));
-    const float nm = -x.mi[0] * kLog2e;
-    const float2 e1 = exp_shift2<T>(zc[0], x.mi[0], l2e2, make_float2(nm, nm));
-    const float2 eT = x.t_one ? e1 : exp_temp2<T>(zc[0], x.mi[0], x.inv_T, kLog2e * x.inv_T);
+    const float2 e1 = exp_from_nml<T>(zc[0], x.nml[0]);
+    const float2 eT = x.t_one ? e1 : exp_temp2<T>(zc[0], m0, x.inv_T, kLog2e * x.inv_T);
     const float2 pT = __fmul2_rn(eT, make_float2(x.cti[0], x.cti[0]));
-    const float2 x0 = __fadd2_rn(zc[0], make_float2(-x.mi[0], -x.mi[0]));
+    const float2 x0 = __fadd2_rn(zc[0], make_float2(-m0, -m0));
     const float2 lp = __ffma2_rn(x0, make_float2(x.inv_T, x.inv_T), make_float2(-x.lsi[0], -x.lsi[0]));
-    const float2 tb = inside(__fmul2_rn(exp_temp2<T>(zb, x.mb, x.inv_T, kLog2e * x.inv_T), make_float2(x.cti[N], x.cti[N])));
+    const float2 tb = __fmul2_rn(exp_temp2<T>(zb, x.mb, x.inv_T, kLog2e * x.inv_T), make_float2(x.cti[N], x.cti[N]));
     const float2 xb = __fadd2_rn(zb, make_float2(-x.mb, -x.mb));
     const float2 lb = __ffma2_rn(xb, make_float2(x.inv_T, x.inv_T), make_float2(-x.lsi[N], -x.lsi[N]));
     const float2 dl = make_float2(fmaxf(lb.x, -3.0e38f) - fmaxf(lp.x, -3.0e38f), fmaxf(lb.y, -3.0e38f) - fmaxf(lp.y, -3.0e38f));
     gc[0] = __ffma2_rn(make_float2(x.ckl, x.ckl), __fadd2_rn(pT, make_float2(-tb.x, -tb.y)),
                        __ffma2_rn(e1, make_float2(x.cpi[0], x.cpi[0]), ncq));
-    acc.dist2[0] = __ffma2_rn(tb, dl, acc.dist2[0]);
+    acc.dist2[0] = __ffma2_rn(counted(tb), dl, acc.dist2[0]);
   }
+}
+
+// One segment off the fast path, element by element: a ragged segment (columns outside the row contribute nothing
+// and are not written), or -- with `count` false -- the segment that holds the label column, whose gradient
+// elements are written once more with the label's term (the fast path wrote them without it).
+// (context and sums in and out by value, so that the caller's copies stay in registers)
+template <typename T, int N, int MODE, bool ALL, int NS>
+__device__ __noinline__ ClColAcc<ALL ? N : 1> cl_slow_segment(ClColCtx<N, NS> x, ClColAcc<ALL ? N : 1> acc, const char* slices, uint32_t slice_bytes,
+                                                              int q, int64_t cbase, int64_t C, bool count, bool only_label, void* const* grad,
+                                                              int64_t img_off, int s) {
+  constexpr int H = SegOps<T>::H;
+  constexpr int NOUT = ALL ? N : 1;
+#pragma unroll 1
+  for (int h = 0; h < H; ++h) {
+    float2 zc[N], gc[NOUT];
+    const int64_t c0 = cbase + 2 * h;
+    const bool in0 = c0 >= 0 && c0 < C, in1 = c0 + 1 >= 0 && c0 + 1 < C;
+    const bool st0 = in0 && (!only_label || c0 == (int64_t)x.y), st1 = in1 && (!only_label || c0 + 1 == (int64_t)x.y);
+    if (!st0 && !st1 && !(count && (in0 || in1))) continue;
+#pragma unroll
+    for (int i = 0; i < N; ++i) {
+      const T* el = reinterpret_cast<const T*>(slices + (size_t)i * slice_bytes + (size_t)q * 16) + 2 * h;
+      const float mi = x.stat[i].m;
+      zc[i] = make_float2(in0 ? Elem<T>::to_f32(el[0]) : mi, in1 ? Elem<T>::to_f32(el[1]) : mi);
+    }
+    cl_column2<T, N, MODE, ALL, true, true>(x, acc, zc, gc, c0, make_float2(count && in0 ? 1.f : 0.f, count && in1 ? 1.f : 0.f));
+#pragma unroll
+    for (int i = 0; i < NOUT; ++i) {
+      if (grad[i] == nullptr) continue;
+      T* ge = reinterpret_cast<T*>(reinterpret_cast<char*>(grad[i]) + img_off + (size_t)s * 16) + 2 * h;
+      if (st0) ge[0] = Elem<T>::from_f32(gc[i].x);
+      if (st1) ge[1] = Elem<T>::from_f32(gc[i].y);
+    }
+  }
+  return acc;
 }
 
 // ------------------------------------------------------------------ the kernel
@@ -338,6 +411,7 @@ __global__ void __launch_bounds__(kClThreads, 2) rows_cluster_kernel(const __gri
   const float inv_T = KL ? 1.f / a.temperature : 1.f;
   const bool t_one = !KL || a.temperature == 1.f;
   const bool need_z = a.eps != 0.f || a.centred != 0;   // sum_c z_c enters the smoothed task loss and the class means
+  const bool want_grad = a.grad[0] != nullptr;
 
   if (tid == 0) {
     for (int i = 0; i < N; ++i) mbar_init(&ctrl->full[i], 1);
@@ -365,6 +439,9 @@ __global__ void __launch_bounds__(kClThreads, 2) rows_cluster_kernel(const __gri
   cx.t_one = t_one;
   cx.centred = a.centred != 0;
   cx.mb = 0.f;
+  cx.stat = ctrl->stat;
+  cx.inv_C = inv_C;
+  cx.cmean = 0.f;
   const int seg_begin = rank * a.spc;
 
   auto row_is_valid = [&](long long r) {
@@ -437,20 +514,25 @@ __global__ void __launch_bounds__(kClThreads, 2) rows_cluster_kernel(const __gri
     const RowGeom g = row_geom<T>(lr, a.row_stride, C);
     const int seg_end = min(seg_begin + a.spc, g.n_seg);
     const int nseg = seg_end > seg_begin ? seg_end - seg_begin : 0;     // segments of this CTA's range in this row
+    // of which [q_lo, q_hi) are whole segments inside the row; a ragged first / last segment of the row image is
+    // done apart by one thread (tid 0 / tid 32)
+    const int q_lo = (seg_begin < g.seg_lo && nseg > 0) ? g.seg_lo - seg_begin : 0;
+    const int q_hi = seg_end > g.seg_hi ? (g.seg_hi > seg_begin ? g.seg_hi - seg_begin : 0) : nseg;
+    const bool edge_head = tid == 0 && q_lo > 0;
+    const bool edge_tail = tid == 32 && q_hi < nseg && q_hi >= q_lo;
+    const int q_edge = edge_head ? 0 : nseg - 1;
     const int64_t img_off = (lr * a.row_stride - g.head) * ES;
     const int y = a.labels[r];
     const bool valid = (a.mask == nullptr || a.mask[r] != 0) && y >= 0 && (int64_t)y < C;
 
     if (!valid) {  // masked row: zero gradient rows, no loss, no counts; nothing is read
+      if (want_grad) {
 #pragma unroll 1
-      for (int i = 0; i < NOUT; ++i) {
-        if (a.grad[i] == nullptr) continue;
-        char* g_img = reinterpret_cast<char*>(a.grad[i]) + img_off;
-        for (int q = tid; q < nseg; q += NT) {
-          const int s = seg_begin + q;
-          if (s >= g.seg_lo && s < g.seg_hi) {
-            *reinterpret_cast<uint4*>(g_img + (size_t)s * 16) = make_uint4(0u, 0u, 0u, 0u);
-          } else {
+        for (int i = 0; i < NOUT; ++i) {
+          char* g_img = reinterpret_cast<char*>(a.grad[i]) + img_off;
+          for (int q = q_lo + tid; q < q_hi; q += NT) *reinterpret_cast<uint4*>(g_img + (size_t)(seg_begin + q) * 16) = make_uint4(0u, 0u, 0u, 0u);
+          if (edge_head || edge_tail) {
+            const int s = seg_begin + q_edge;
 #pragma unroll
             for (int e = 0; e < V; ++e) {
               const int64_t c = (int64_t)s * V - g.head + e;
@@ -469,29 +551,54 @@ __global__ void __launch_bounds__(kClThreads, 2) rows_cluster_kernel(const __gri
     // Every warp takes a share of each tensor, so the sweep of tensor i runs while tensors i+1.. are still
     // in flight.  One lane per warp watches the copy barrier (with back-off): waiting warps take next to no
     // issue slots from the CTA that shares the SM.
-#pragma unroll 1
-    for (int i = 0; i < N; ++i) {
-      if (lane == 0) cl_wait(&ctrl->full[i], (uint32_t)v & 1u, ctrl, a.hdr);
-      __syncwarp();
-      const char* sl = slices + (size_t)i * a.slice_bytes;
-      ClAcc<H> acc;
-      acc.reset();
-      for (int q = tid; q < nseg; q += NT) {
-        const int s = seg_begin + q;
-        const uint4 raw = *reinterpret_cast<const uint4*>(sl + (size_t)q * 16);
-        if (s >= g.seg_lo && s < g.seg_hi) {
-          if (t_one) cl_sweep_seg<T, false>(acc, raw, s, inv_T, need_z); else cl_sweep_seg<T, KL>(acc, raw, s, inv_T, need_z);
-        } else {
-          acc = t_one ? cl_sweep_edge<T, false>(acc, raw, s, g.head, C, inv_T) : cl_sweep_edge<T, KL>(acc, raw, s, g.head, C, inv_T);
+    {
+      ClLane L[N];
+#pragma unroll
+      for (int i = 0; i < N; ++i) {
+        if (lane == 0) cl_wait(&ctrl->full[i], (uint32_t)v & 1u, ctrl, a.hdr);
+        __syncwarp();
+        const char* sl = slices + (size_t)i * a.slice_bytes;
+        L[i] = t_one ? cl_sweep_range<T, false>(sl, q_lo, q_hi, seg_begin, tid, inv_T, need_z)
+                     : cl_sweep_range<T, KL>(sl, q_lo, q_hi, seg_begin, tid, inv_T, need_z);
+        if (edge_head || edge_tail) {
+          const uint4 raw = *reinterpret_cast<const uint4*>(sl + (size_t)q_edge * 16);
+          L[i] = t_one ? cl_sweep_edge<T, false>(L[i], raw, seg_begin + q_edge, g.head, C, inv_T)
+                       : cl_sweep_edge<T, KL>(L[i], raw, seg_begin + q_edge, g.head, C, inv_T);
         }
       }
-      const ClRec rec = t_one ? cl_warp_record<T, false>(acc, i, inv_T) : cl_warp_record<T, KL>(acc, i, inv_T);
-      if (lane == 0) ctrl->rec[warp][i] = rec;
+      // per tensor the warp's maximum and its first segment by integer reductions; then all the sums at once
+      constexpr int NQ = KL ? 3 : 2;
+      constexpr int NV = cl_pow2_at_least(NQ * N);
+      float vals[NV];
+#pragma unroll
+      for (int k = 0; k < NV; ++k) vals[k] = 0.f;
+#pragma unroll
+      for (int i = 0; i < N; ++i) {
+        const unsigned key = float_order_key(L[i].best + 0.f);   // -0 is folded onto +0: they tie
+        const unsigned key_w = __reduce_max_sync(0xffffffffu, key);
+        const int seg_w = (int)__reduce_min_sync(0xffffffffu, key == key_w ? (unsigned)L[i].seg : 0x7fffffffu);
+        const float m_w = float_from_order_key(key_w);
+        vals[i] = L[i].s * rescale_exp2<T>((L[i].best - m_w) * kLog2e);
+        vals[N + i] = L[i].z;
+        if constexpr (KL) vals[2 * N + i] = t_one ? 0.f : L[i].t * rescale_exp2<T>((L[i].best - m_w) * (kLog2e * inv_T));
+        if (lane == 0) { ctrl->rec[warp][i].m = m_w; ctrl->rec[warp][i].seg = seg_w; }
+      }
+      warp_multi_sum<NV>(vals, lane);
+      constexpr int kShift = 5 - cl_log2(NV);
+      if ((lane & ((1 << kShift) - 1)) == 0) {
+        const int j = lane >> kShift;
+        if (j < NQ * N) {
+          const int quantity = j / N, i = j - quantity * N;
+          if (quantity == 0) ctrl->rec[warp][i].S = vals[0];
+          else if (quantity == 1) ctrl->rec[warp][i].sum_z = vals[0];
+          else ctrl->rec[warp][i].S_T = vals[0];
+        }
+      }
     }
     if constexpr (KLM) {
       // statistics of the averaged peer logits zbar = mean_{j >= 1} z_j at temperature T
-      ClAcc<H> acc;
-      acc.reset();
+      ClLane L;
+      L.best = -3.0e38f; L.seg = 0x7fffffff; L.s = 0.f; L.z = 0.f; L.t = 0.f;
       const float inv_P = 1.f / (float)(N - 1);
       for (int q = tid; q < nseg; q += NT) {
         const int s = seg_begin + q;
@@ -518,16 +625,19 @@ __global__ void __launch_bounds__(kClThreads, 2) rows_cluster_kernel(const __gri
           if (in[2 * h]) fm = fmaxf(fm, zb[h].x);
           if (in[2 * h + 1]) fm = fmaxf(fm, zb[h].y);
         }
-        cl_raise<T, true>(acc, fm, s, inv_T);
+        const float nb = fmaxf(L.best, fm);
+        L.t *= rescale_exp2<T>((L.best - nb) * (kLog2e * inv_T));
+        L.best = nb;
 #pragma unroll
         for (int h = 0; h < H; ++h) {
-          const float2 e2 = exp_temp2<T>(zb[h], acc.best, inv_T, kLog2e * inv_T);
-          if (in[2 * h]) acc.t2[h].x += e2.x;
-          if (in[2 * h + 1]) acc.t2[h].y += e2.y;
+          const float2 e2 = exp_temp2<T>(zb[h], nb, inv_T, kLog2e * inv_T);
+          if (in[2 * h]) L.t += e2.x;
+          if (in[2 * h + 1]) L.t += e2.y;
         }
       }
-      const ClRec rec = cl_warp_record<T, true>(acc, N, inv_T);
-      if (lane == 0) ctrl->rec[warp][N] = rec;
+      const float m_w = warp_max_redux(L.best);
+      const float t_w = warp_sum(L.t * rescale_exp2<T>((L.best - m_w) * (kLog2e * inv_T)));
+      if (lane == 0) { ClRec rc; rc.m = m_w; rc.seg = 0x7fffffff; rc.S = 0.f; rc.sum_z = 0.f; rc.S_T = t_w; rc.tensor = N; ctrl->rec[warp][N] = rc; }
     }
     __syncthreads();
     // This CTA's partial result of tensor i, by warp i: one warp's record per lane (the first segment that attains
@@ -552,9 +662,7 @@ __global__ void __launch_bounds__(kClThreads, 2) rows_cluster_kernel(const __gri
           }
         }
         const int seg_y = (g.head + y) / V;
-        if (seg_y >= seg_begin && seg_y < seg_end) {
-          p.zy = Elem<T>::to_f32(sl[(size_t)(seg_y - seg_begin) * V + (g.head + y) % V]);
-        }
+        if (seg_y >= seg_begin && seg_y < seg_end) p.zy = Elem<T>::to_f32(sl[(size_t)(seg_y - seg_begin) * V + (g.head + y) % V]);
       }
       if (lane < K) *cluster.map_shared_rank(&ctrl->gather[par][rank][i], lane) = p;
     }
@@ -578,17 +686,17 @@ __global__ void __launch_bounds__(kClThreads, 2) rows_cluster_kernel(const __gri
       ctrl->pend[par][tid] = ctrl->stat[tid];
       if (tid == 0) { ctrl->pend_row[par] = r; ctrl->pend_y[par] = y; }
     }
-    float class_mean_avg = 0.f;
+    {
+      float cm = 0.f;
 #pragma unroll
-    for (int i = 0; i < N; ++i) class_mean_avg += ctrl->stat[i].sum_z;
-    class_mean_avg *= inv_C / (float)N;
-#pragma unroll
-    for (int i = 0; i < N; ++i) {
-      const ClStat st = ctrl->stat[i];
-      cx.mi[i] = st.m;
-      cx.cpi[i] = w * __frcp_rn(st.S);
-      cx.cmi[i] = class_mean_avg - st.sum_z * inv_C;
-      if constexpr (KL) { cx.cti[i] = __frcp_rn(st.S_T); cx.lsi[i] = logf(st.S_T); }
+      for (int i = 0; i < N; ++i) {
+        const ClStat st = ctrl->stat[i];
+        cx.nml[i] = ES == 4 ? -st.m : -st.m * kLog2e;
+        cx.cpi[i] = w * __frcp_rn(st.S);
+        cm += st.sum_z;
+        if constexpr (KL) { cx.cti[i] = __frcp_rn(st.S_T); cx.lsi[i] = logf(st.S_T); }
+      }
+      cx.cmean = cm * inv_C / (float)N;
     }
     if constexpr (KLM) { const ClStat st = ctrl->stat[N]; cx.mb = st.m; cx.cti[N] = __frcp_rn(st.S_T); cx.lsi[N] = logf(st.S_T); }
     cx.y = y;
@@ -598,82 +706,76 @@ __global__ void __launch_bounds__(kClThreads, 2) rows_cluster_kernel(const __gri
     acc.qs2 = make_float2(0.f, 0.f);
 #pragma unroll
     for (int i = 0; i < NOUT; ++i) acc.dist2[i] = make_float2(0.f, 0.f);
-    const int seg_y = (g.head + y) / V;
-    for (int q = tid; q < nseg; q += NT) {
+#pragma unroll 1
+    for (int q = q_lo + tid; q < q_hi; q += NT) {
       const int s = seg_begin + q;
       const int64_t cbase = (int64_t)s * V - g.head;
-      const bool lab = s == seg_y;
       uint4 rw[N];
 #pragma unroll
       for (int i = 0; i < N; ++i) rw[i] = *reinterpret_cast<const uint4*>(slices + (size_t)i * a.slice_bytes + (size_t)q * 16);
-      if (s >= g.seg_lo && s < g.seg_hi) {
 #pragma unroll
-        for (int h = 0; h < H; ++h) {
-          float2 zc[N], gc[NOUT];
+      for (int h = 0; h < H; ++h) {
+        float2 zc[N], gc[NOUT];
 #pragma unroll
-          for (int i = 0; i < N; ++i) {
-            if constexpr (ES == 4) {
-              zc[i] = h == 0 ? make_float2(__uint_as_float(rw[i].x), __uint_as_float(rw[i].y))
-                             : make_float2(__uint_as_float(rw[i].z), __uint_as_float(rw[i].w));
-            } else {
-              const uint32_t word = h == 0 ? rw[i].x : h == 1 ? rw[i].y : h == 2 ? rw[i].z : rw[i].w;
-              zc[i] = make_float2(__uint_as_float(word << 16), __uint_as_float(word & 0xFFFF0000u));
-            }
-          }
-          cl_column2<T, N, MODE, ALL, false>(cx, acc, zc, gc, cbase + 2 * h, lab, make_float2(1.f, 1.f));
-#pragma unroll
-          for (int i = 0; i < NOUT; ++i) {
-            if constexpr (ES == 4) {
-              if (h == 0) { rw[i].x = __float_as_uint(gc[i].x); rw[i].y = __float_as_uint(gc[i].y); }
-              else { rw[i].z = __float_as_uint(gc[i].x); rw[i].w = __float_as_uint(gc[i].y); }
-            } else {
-              const __nv_bfloat162 pk = __floats2bfloat162_rn(gc[i].x, gc[i].y);
-              const uint32_t word = *reinterpret_cast<const uint32_t*>(&pk);
-              if (h == 0) rw[i].x = word; else if (h == 1) rw[i].y = word; else if (h == 2) rw[i].z = word; else rw[i].w = word;
-            }
+        for (int i = 0; i < N; ++i) {
+          if constexpr (ES == 4) {
+            zc[i] = h == 0 ? make_float2(__uint_as_float(rw[i].x), __uint_as_float(rw[i].y))
+                           : make_float2(__uint_as_float(rw[i].z), __uint_as_float(rw[i].w));
+          } else {
+            const uint32_t word = h == 0 ? rw[i].x : h == 1 ? rw[i].y : h == 2 ? rw[i].z : rw[i].w;
+            zc[i] = make_float2(__uint_as_float(word << 16), __uint_as_float(word & 0xFFFF0000u));
           }
         }
+        cl_column2<T, N, MODE, ALL, false, false>(cx, acc, zc, gc, cbase + 2 * h, make_float2(1.f, 1.f));
 #pragma unroll
-        for (int i = 0; i < NOUT; ++i)
-          if (a.grad[i] != nullptr) *reinterpret_cast<uint4*>(reinterpret_cast<char*>(a.grad[i]) + img_off + (size_t)s * 16) = rw[i];
-      } else {
-        // ragged segment: same arithmetic, columns outside the row contribute nothing and are not written
-#pragma unroll 1
-        for (int h = 0; h < H; ++h) {
-          float2 zc[N], gc[NOUT];
-          const int64_t c0 = cbase + 2 * h;
-          const bool in0 = c0 >= 0 && c0 < C, in1 = c0 + 1 >= 0 && c0 + 1 < C;
-#pragma unroll
-          for (int i = 0; i < N; ++i) {
-            const T* el = reinterpret_cast<const T*>(slices + (size_t)i * a.slice_bytes + (size_t)q * 16) + 2 * h;
-            zc[i] = make_float2(in0 ? Elem<T>::to_f32(el[0]) : cx.mi[i], in1 ? Elem<T>::to_f32(el[1]) : cx.mi[i]);
-          }
-          cl_column2<T, N, MODE, ALL, true>(cx, acc, zc, gc, c0, lab, make_float2(in0 ? 1.f : 0.f, in1 ? 1.f : 0.f));
-#pragma unroll
-          for (int i = 0; i < NOUT; ++i) {
-            if (a.grad[i] == nullptr) continue;
-            T* ge = reinterpret_cast<T*>(reinterpret_cast<char*>(a.grad[i]) + img_off + (size_t)s * 16) + 2 * h;
-            if (in0) ge[0] = Elem<T>::from_f32(gc[i].x);
-            if (in1) ge[1] = Elem<T>::from_f32(gc[i].y);
+        for (int i = 0; i < NOUT; ++i) {
+          if constexpr (ES == 4) {
+            if (h == 0) { rw[i].x = __float_as_uint(gc[i].x); rw[i].y = __float_as_uint(gc[i].y); }
+            else { rw[i].z = __float_as_uint(gc[i].x); rw[i].w = __float_as_uint(gc[i].y); }
+          } else {
+            const __nv_bfloat162 pk = __floats2bfloat162_rn(gc[i].x, gc[i].y);
+            const uint32_t word = *reinterpret_cast<const uint32_t*>(&pk);
+            if (h == 0) rw[i].x = word; else if (h == 1) rw[i].y = word; else if (h == 2) rw[i].z = word; else rw[i].w = word;
           }
         }
       }
+      if (want_grad) {
+#pragma unroll
+        for (int i = 0; i < NOUT; ++i) *reinterpret_cast<uint4*>(reinterpret_cast<char*>(a.grad[i]) + img_off + (size_t)s * 16) = rw[i];
+      }
+    }
+    // the ragged segments, element by element
+    if (edge_head || edge_tail)
+      acc = cl_slow_segment<T, N, MODE, ALL>(cx, acc, slices, a.slice_bytes, q_edge, (int64_t)(seg_begin + q_edge) * V - g.head, C, true, false,
+                                       a.grad, img_off, seg_begin + q_edge);
+    // the label column: its gradient elements once more, now with the label's term (a label inside a ragged segment
+    // has had it already).  The thread that wrote the segment above writes it again: its stores stay in order.
+    {
+      const int seg_y = (g.head + y) / V;
+      const int qy = seg_y - seg_begin;
+      if (want_grad && qy >= q_lo && qy < q_hi && (qy - q_lo) % NT == tid)
+        acc = cl_slow_segment<T, N, MODE, ALL>(cx, acc, slices, a.slice_bytes, qy, (int64_t)seg_y * V - g.head, C, false, true, a.grad, img_off, seg_y);
     }
 
     // ================= distance partial sums of this CTA, handed to CTA 0 (which reads them behind the next cluster barrier)
+    {
+      constexpr int ND = cl_pow2_at_least(NOUT + 1);
+      float dv[ND];
 #pragma unroll
-    for (int i = 0; i < NOUT; ++i) {
-      const float dw = warp_sum(acc.dist2[i].x + acc.dist2[i].y);
-      if (lane == 0) ctrl->dwarp[warp][i] = dw;
-    }
-    if constexpr (MODE == kClMse) {
+      for (int k = 0; k < ND; ++k) dv[k] = 0.f;
       float qt = acc.qs2.x + acc.qs2.y;
-      if constexpr (ALL) {
 #pragma unroll
-        for (int i = 0; i < N; ++i) qt += acc.dist2[i].x + acc.dist2[i].y;
+      for (int i = 0; i < NOUT; ++i) {
+        dv[i] = acc.dist2[i].x + acc.dist2[i].y;
+        if constexpr (ALL) qt += dv[i];
       }
-      const float qw = warp_sum(qt);
-      if (lane == 0) ctrl->dwarp[warp][kClMax] = qw;
+      dv[NOUT] = MODE == kClMse ? qt : 0.f;
+      warp_multi_sum<ND>(dv, lane);
+      constexpr int kShiftD = 5 - cl_log2(ND);
+      if ((lane & ((1 << kShiftD) - 1)) == 0) {
+        const int j = lane >> kShiftD;
+        if (j <= NOUT) ctrl->dwarp[warp][j == NOUT ? kClMax : j] = dv[0];
+      }
     }
     __syncthreads();   // pass B has read the ranges: they may be overwritten; the warps' partial sums are in place
     if (tid == 0) {
@@ -685,10 +787,8 @@ __global__ void __launch_bounds__(kClThreads, 2) rows_cluster_kernel(const __gri
     if (tid >= 32 && tid - 32 <= kClMax && (tid - 32 < NOUT || tid - 32 == kClMax)) {
       const int i = tid - 32;
       float d = 0.f;
-      if (i < NOUT || MODE == kClMse) {
 #pragma unroll
-        for (int wv = 0; wv < NW; ++wv) d += ctrl->dwarp[wv][i];
-      }
+      for (int wv = 0; wv < NW; ++wv) d += ctrl->dwarp[wv][i];
       *cluster.map_shared_rank(&ctrl->dgather[par][rank][i], 0) = d;
     }
     ++v;

@@ -1,7 +1,9 @@
 """GPU parity of the cluster-resident kernel (all n row images of a row index kept in the shared memory
 of a thread-block cluster): every cluster size, both call forms (single model / all models), every
 distance it serves, rows that straddle the CTAs' column ranges in all the awkward ways (unaligned rows,
-ragged first and last segments, ranges that end up empty), planted maxima on range boundaries."""
+ragged first and last segments, ranges that end up empty), planted maxima on range boundaries.  The kernel
+is asked for through CODISTILL_REGIME=cluster; by default it serves only the peer counts the other long-row
+kernels are not built for."""
 import numpy as np
 import pytest
 import torch
@@ -31,6 +33,7 @@ def rand_models(seed, rows, C, n, dtype, scale=1.5, spread=0.7):
 
 @pytest.fixture(params=[1, 2, 4, 8, 16])
 def cluster_size(request, monkeypatch):
+    monkeypatch.setenv("CODISTILL_REGIME", "cluster")
     monkeypatch.setenv("CODISTILL_CLUSTER_SIZE", str(request.param))
     return request.param
 
@@ -52,8 +55,7 @@ def test_single_model_call_every_cluster_size(cluster_size, n, C, dtype):
 
 
 @pytest.mark.parametrize("n,C,dtype", [(2, 8192, "bf16"), (8, 5003, "bf16"), (3, 4099, "f32")])
-def test_plain_mse_on_request(cluster_size, monkeypatch, n, C, dtype):
-    monkeypatch.setenv("CODISTILL_REGIME", "cluster")
+def test_plain_mse_on_request(cluster_size, n, C, dtype):
     rows = 150
     models, labels, mask = rand_models(37 * n + C, rows, C, n, dtype)
     for pr in (cb.PEERS_PAIRWISE_MEAN, cb.PEERS_MEAN_TARGET):
@@ -76,14 +78,15 @@ def test_all_models_call_every_cluster_size(cluster_size, n, C, dtype):
 
 @pytest.mark.parametrize("n", [5, 6, 7])
 @pytest.mark.parametrize("dtype", ["f32", "bf16"])
-def test_plain_mse_with_four_to_six_peers_stays_on_a_long_row_kernel(n, dtype):
-    """The staged and direct-load MSE kernels are built for 0-3 and 7 peers; the peer counts between are
-    served by the cluster-resident kernel, not by the one-CTA-per-row fallback."""
+def test_four_to_six_peers_stay_on_a_long_row_kernel(n, dtype):
+    """The staged and direct-load kernels are built for 0-3 and 7 peers; the peer counts between are served by
+    the cluster-resident kernel (by default), not by the one-CTA-per-row fallback."""
     rows, C = 300, 9001 if dtype == "bf16" else 4099
     models, labels, mask = rand_models(43 * n, rows, C, n, dtype)
-    for pr in (cb.PEERS_PAIRWISE_MEAN, cb.PEERS_MEAN_TARGET):
-        compare(models[0], models[1:], labels, mask, alpha=0.9, label_smoothing=0.05, peer_reduce=pr,
-                reduction=cb.REDUCE_SUM, expect_regime="cluster")
+    for dist, pr in ((cb.DIST_MSE_LOGITS, cb.PEERS_PAIRWISE_MEAN), (cb.DIST_MSE_LOGITS, cb.PEERS_MEAN_TARGET),
+                     (cb.DIST_KL_SOFTMAX, cb.PEERS_PAIRWISE_MEAN), (cb.DIST_MSE_CENTRED, cb.PEERS_PAIRWISE_MEAN)):
+        compare(models[0], models[1:], labels, mask, alpha=0.9, temperature=1.5, label_smoothing=0.05, dist=dist,
+                peer_reduce=pr, reduction=cb.REDUCE_SUM, expect_regime="cluster")
 
 
 @pytest.mark.parametrize("dtype", ["f32", "bf16"])
@@ -122,9 +125,10 @@ def test_maxima_on_range_boundaries(cluster_size, dtype):
     compare_all(models, labels, None, alpha=1.0, reduction=cb.REDUCE_SUM)
 
 
-def test_guard_bands_and_determinism():
+def test_guard_bands_and_determinism(monkeypatch):
     """Nothing is written outside the gradient rows (an unaligned last row ends inside a 16-byte segment),
     two runs are bit-identical, inputs are left alone."""
+    monkeypatch.setenv("CODISTILL_REGIME", "cluster")
     rows, C, n = 40, 9001, 4
     models, labels, mask = rand_models(9, rows, C, n, "bf16")
     keep = [m.copy() for m in models]

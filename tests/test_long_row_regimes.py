@@ -92,24 +92,23 @@ def test_very_long_rows_take_the_stream_kernel():
 @pytest.mark.parametrize("peer_reduce", [cb.PEERS_PAIRWISE_MEAN, cb.PEERS_MEAN_TARGET])
 @pytest.mark.parametrize("C,n,temperature", [(32768, 2, 1.0), (50257, 4, 2.0), (9001, 8, 0.7), (8192, 1, 3.0)])
 def test_kl_form_on_long_rows(dtype, peer_reduce, C, n, temperature):
-    """The softmax-KL distance on long rows: with peers the cluster-resident kernel (all n rows on chip),
-    without them the direct-load kernel."""
+    """The softmax-KL distance on long rows is served by the direct-load kernel (one more pass for the
+    peers' softmax statistics)."""
     rows = 13
     own, peers, labels = rand_inputs(3 * C + n, rows, C, n, dtype)
     mask = (np.arange(rows) % 5 != 3).astype(np.uint8)
     labels[0], labels[1] = 0, C - 1
     for reduction in (cb.REDUCE_SUM, cb.REDUCE_MEAN_VALID):
         compare(own, peers, labels, mask, alpha=0.9, temperature=temperature, label_smoothing=0.05,
-                dist=cb.DIST_KL_SOFTMAX, peer_reduce=peer_reduce, reduction=reduction,
-                expect_regime="cluster" if n > 1 else "stream")
+                dist=cb.DIST_KL_SOFTMAX, peer_reduce=peer_reduce, reduction=reduction, expect_regime="stream")
 
 
 @pytest.mark.parametrize("dtype", ["f32", "bf16"])
 @pytest.mark.parametrize("peer_reduce", [cb.PEERS_PAIRWISE_MEAN, cb.PEERS_MEAN_TARGET])
 @pytest.mark.parametrize("C,n", [(32768, 2), (50257, 4), (9001, 8), (8192, 1)])
 def test_centred_mse_on_long_rows(dtype, peer_reduce, C, n):
-    """The centred MSE distance on long rows: with peers the cluster-resident kernel, without them the
-    direct-load kernel."""
+    """The centred MSE distance on long rows is served by the direct-load kernel (one more pass for the
+    peers' class sums)."""
     rows = 13
     own, peers, labels = rand_inputs(5 * C + n, rows, C, n, dtype)
     peers = [p if p.dtype == np.uint16 else (p + np.float32(0.5 * (j + 1))) for j, p in enumerate(peers)]  # shifted peers
@@ -117,17 +116,4 @@ def test_centred_mse_on_long_rows(dtype, peer_reduce, C, n):
     labels[0], labels[1] = 0, C - 1
     for reduction in (cb.REDUCE_SUM, cb.REDUCE_MEAN_VALID):
         compare(own, peers, labels, mask, alpha=0.9, label_smoothing=0.05, dist=cb.DIST_MSE_CENTRED,
-                peer_reduce=peer_reduce, reduction=reduction, expect_regime="cluster" if n > 1 else "stream")
-
-
-@pytest.mark.parametrize("dist", [cb.DIST_KL_SOFTMAX, cb.DIST_MSE_CENTRED])
-@pytest.mark.parametrize("C,n,temperature", [(32768, 2, 1.0), (9001, 4, 2.0), (9001, 8, 0.7)])
-def test_direct_load_kernels_serve_kl_and_centred_on_request(monkeypatch, dist, C, n, temperature):
-    """The direct-load kernels remain the path for rows too long to keep on chip; here they are asked for."""
-    monkeypatch.setenv("CODISTILL_REGIME", "stream")
-    rows = 13
-    own, peers, labels = rand_inputs(7 * C + n, rows, C, n, "bf16")
-    mask = (np.arange(rows) % 5 != 3).astype(np.uint8)
-    for peer_reduce in (cb.PEERS_PAIRWISE_MEAN, cb.PEERS_MEAN_TARGET):
-        compare(own, peers, labels, mask, alpha=0.9, temperature=temperature, label_smoothing=0.05, dist=dist,
-                peer_reduce=peer_reduce, reduction=cb.REDUCE_SUM, expect_regime="stream")
+                peer_reduce=peer_reduce, reduction=reduction, expect_regime="stream")

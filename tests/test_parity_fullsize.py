@@ -87,7 +87,10 @@ def all_models_call(idx, dist):
     kw = dict(alpha=w.alpha, temperature=w.temperature, label_smoothing=w.label_smoothing, dist=DIST[dist])
     counters, losses, row_loss = out.counters.cpu().numpy(), out.loss.cpu().numpy(), out.row_loss.cpu().numpy()
     R = w.rows
-    for i in range(w.n):
+    # every model of a small ensemble; of a large one the first, a middle and the last model (the oracle needs
+    # a whole pass over all n tensors per model checked)
+    checked = range(w.n) if w.n <= 4 else (0, w.n // 2, w.n - 1)
+    for i in checked:
         peers = models[:i] + models[i + 1:]
         ref = oracle.codistill(models[i], peers, labels, mask, want_grad=False, **kw)
         assert counters[i].tolist() == ref.counters.tolist()
