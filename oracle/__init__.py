@@ -20,7 +20,7 @@ _SRC = os.path.join(_HERE, "codistill_oracle.c")
 _SO = os.path.join(_HERE, "liboracle.so")
 
 F32, BF16 = 0, 1
-DIST_MSE, DIST_KL, DIST_MSE_CENTRED = 0, 1, 2
+DIST_MSE, DIST_KL, DIST_MSE_CENTRED, DIST_KL_REVERSE, DIST_KL_SYMMETRIC = 0, 1, 2, 3, 4
 PEERS_PAIRWISE, PEERS_MEAN_TARGET = 0, 1
 REDUCE_MEAN_VALID, REDUCE_SUM = 0, 1
 

@@ -16,6 +16,8 @@
  *     the two models, not centred; the same passage says that centring the logits gave similar
  *     results: the centred variant (each model's logits minus their mean over the classes before the
  *     squared error, i.e. the variance over the classes of the difference) is dist_kind 2.
+ *   - Section 2 does not fix the direction of the KL divergence; the peer-as-target direction is dist_kind 1,
+ *     the other direction dist_kind 3 and their average dist_kind 4.
  *   - Section 3 / Section 5: the term may be omitted (non-communication steps), n = 1 is
  *     ordinary training.
  * Readings where the paper is silent: label smoothing is uniform, q = (1 - eps) onehot(y) + eps / C;
@@ -40,7 +42,9 @@
 #endif
 
 enum { ORACLE_F32 = 0, ORACLE_BF16 = 1 };
-enum { ORACLE_DIST_MSE = 0, ORACLE_DIST_KL = 1, ORACLE_DIST_MSE_CENTRED = 2 };
+enum { ORACLE_DIST_MSE = 0, ORACLE_DIST_KL = 1, ORACLE_DIST_MSE_CENTRED = 2,
+       ORACLE_DIST_KL_REVERSE = 3,   /* T^2 KL(softmax(own / T) || softmax(peer / T)): the other direction of Section 2's KL */
+       ORACLE_DIST_KL_SYMMETRIC = 4  /* half the sum of the two directions */ };
 enum { ORACLE_PEERS_PAIRWISE = 0, ORACLE_PEERS_MEAN_TARGET = 1 };
 enum { ORACLE_REDUCE_MEAN_VALID = 0, ORACLE_REDUCE_SUM = 1 };
 enum { ORACLE_STATUS_BAD_LABEL = 1 };
@@ -64,6 +68,34 @@ static double log_sum_exp(const double* v, int64_t C, int64_t* argmax_out) {
   for (int64_t c = 0; c < C; ++c) s += exp(v[c] - m);
   if (argmax_out) *argmax_out = a;
   return m + log(s);
+}
+
+/*
+ * The softmax-KL family between own logits z and target logits v (a peer, or the mean of the peers), both
+ * at temperature T, with p = softmax(z / T), t = softmax(v / T):
+ *   forward  T^2 KL(t || p) = T^2 sum_c t_c (log t_c - log p_c),   d/dz_k = T (p_k - t_k)
+ *   reverse  T^2 KL(p || t) = T^2 sum_c p_c (log p_c - log t_c),   d/dz_k = T p_k ((log p_k - log t_k) - KL(p || t))
+ * weighted by wf and wr (1, 0: forward; 0, 1: reverse; 1/2, 1/2: symmetric).  Returns the weighted value and adds
+ * scale times its derivative to dD.  lse_z = log sum exp(z / T); tmp is scratch of C doubles.
+ */
+static double kl_family(const double* z, const double* v, int64_t C, double T, double lse_z, double wf, double wr,
+                        double scale, double* dD, double* tmp) {
+  for (int64_t c = 0; c < C; ++c) tmp[c] = v[c] / T;
+  const double lse_v = log_sum_exp(tmp, C, NULL);
+  double kl_f = 0.0, kl_r = 0.0;
+  for (int64_t c = 0; c < C; ++c) {
+    const double log_t = v[c] / T - lse_v;
+    const double log_p = z[c] / T - lse_z;
+    kl_f += exp(log_t) * (log_t - log_p);
+    kl_r += exp(log_p) * (log_p - log_t);
+  }
+  for (int64_t c = 0; c < C; ++c) {
+    const double log_t = v[c] / T - lse_v;
+    const double log_p = z[c] / T - lse_z;
+    const double p = exp(log_p), t = exp(log_t);
+    dD[c] += scale * (wf * T * (p - t) + wr * T * p * ((log_p - log_t) - kl_r));
+  }
+  return T * T * (wf * kl_f + wr * kl_r);
 }
 
 /* A row takes part iff its mask byte is non-zero (or there is no mask) and its label is a class id. */
@@ -159,7 +191,10 @@ int codistill_oracle(const void* own, const void* const* peers, const int32_t* l
       for (int64_t c = 0; c < C; ++c) { dD[c] = 0.0; zbar[c] = 0.0; }
       if (P >= 1) {
         double lse_own_T = 0.0;
-        if (dist_kind == ORACLE_DIST_KL) {
+        const int kl_family_kind = dist_kind == ORACLE_DIST_KL || dist_kind == ORACLE_DIST_KL_REVERSE || dist_kind == ORACLE_DIST_KL_SYMMETRIC;
+        const double wf = dist_kind == ORACLE_DIST_KL ? 1.0 : dist_kind == ORACLE_DIST_KL_SYMMETRIC ? 0.5 : 0.0;
+        const double wr = dist_kind == ORACLE_DIST_KL_REVERSE ? 1.0 : dist_kind == ORACLE_DIST_KL_SYMMETRIC ? 0.5 : 0.0;
+        if (kl_family_kind) {
           for (int64_t c = 0; c < C; ++c) tmp[c] = z[c] / T;
           lse_own_T = log_sum_exp(tmp, C, NULL);
         }
@@ -195,18 +230,8 @@ int codistill_oracle(const void* own, const void* const* peers, const int32_t* l
               }
               D += dj / (double)C / (double)P;
             } else {
-              /* D_j = T^2 KL(t^(j) || p^T), t^(j) = softmax(z^(j)/T), p^T = softmax(z/T) */
-              for (int64_t c = 0; c < C; ++c) tmp[c] = zj[c] / T;
-              const double lse_j = log_sum_exp(tmp, C, NULL);
-              double kl = 0.0;
-              for (int64_t c = 0; c < C; ++c) {
-                const double log_t = zj[c] / T - lse_j;
-                const double log_p = z[c] / T - lse_own_T;
-                const double t = exp(log_t);
-                kl += t * (log_t - log_p);
-                dD[c] += T * (exp(log_p) - t) / (double)P;
-              }
-              D += T * T * kl / (double)P;
+              /* D_j = T^2 KL(t^(j) || p^T), t^(j) = softmax(z^(j)/T), p^T = softmax(z/T), or its other direction */
+              D += kl_family(z, zj, C, T, lse_own_T, wf, wr, 1.0 / (double)P, dD, tmp) / (double)P;
             }
           }
         }
@@ -231,17 +256,7 @@ int codistill_oracle(const void* own, const void* const* peers, const int32_t* l
             }
             D = d2 / (double)C;
           } else {
-            for (int64_t c = 0; c < C; ++c) tmp[c] = zbar[c] / T;
-            const double lse_b = log_sum_exp(tmp, C, NULL);
-            double kl = 0.0;
-            for (int64_t c = 0; c < C; ++c) {
-              const double log_t = zbar[c] / T - lse_b;
-              const double log_p = z[c] / T - lse_own_T;
-              const double t = exp(log_t);
-              kl += t * (log_t - log_p);
-              dD[c] = T * (exp(log_p) - t);
-            }
-            D = T * T * kl;
+            D = kl_family(z, zbar, C, T, lse_own_T, wf, wr, 1.0, dD, tmp);
           }
         }
       }

@@ -15,7 +15,8 @@ import oracle
 from paper_2010_02838_b200 import synth
 
 GOLDEN = os.path.join(os.path.dirname(__file__), "golden")
-DISTS = [oracle.DIST_MSE, oracle.DIST_KL, oracle.DIST_MSE_CENTRED]
+DISTS = [oracle.DIST_MSE, oracle.DIST_KL, oracle.DIST_MSE_CENTRED, oracle.DIST_KL_REVERSE, oracle.DIST_KL_SYMMETRIC]
+SHIFT_INVARIANT = (oracle.DIST_KL, oracle.DIST_MSE_CENTRED, oracle.DIST_KL_REVERSE, oracle.DIST_KL_SYMMETRIC)
 PEER_REDUCES = [oracle.PEERS_PAIRWISE, oracle.PEERS_MEAN_TARGET]
 
 
@@ -103,7 +104,7 @@ def test_gradient_row_sums(dist):
     alpha, C = 0.9, 13
     res = oracle.codistill(own, peers, labels, alpha=alpha, temperature=1.5, label_smoothing=0.2, dist=dist,
                            reduction=oracle.REDUCE_SUM)
-    if dist in (oracle.DIST_KL, oracle.DIST_MSE_CENTRED):   # shift-invariant distances: their gradient sums to zero
+    if dist in SHIFT_INVARIANT:   # shift-invariant distances: their gradient sums to zero
         assert res.grad.sum(1) == pytest.approx(np.zeros(4), abs=1e-13)
     else:
         zbar = sum(widen(p) for p in peers) / 3
@@ -151,7 +152,7 @@ def test_shift_behaviour_mse_and_kl():
         assert both.row_loss == pytest.approx(base.row_loss, rel=1e-12)
         assert both.grad == pytest.approx(base.grad, abs=1e-13)
         only_own = oracle.codistill(own_s, peers, labels, alpha=1.1, dist=dist, reduction=oracle.REDUCE_SUM)
-        if dist in (oracle.DIST_KL, oracle.DIST_MSE_CENTRED):   # centring removes a shift of the own logits
+        if dist in SHIFT_INVARIANT:   # centring removes a shift of the own logits
             assert only_own.row_loss == pytest.approx(base.row_loss, rel=1e-12)
         else:  # un-centred MSE: D changes by 2k mean_c(z - zbar) + k^2
             zbar = sum(to64(p) for p in peers) / len(peers)
@@ -177,6 +178,33 @@ def test_kl_form_n2_T1_closed_form_and_one_hot_limit():
     sharp[np.arange(4), cls] = 80.0
     res2 = oracle.codistill(own, [sharp], labels, alpha=1.0, dist=oracle.DIST_KL, reduction=oracle.REDUCE_SUM)
     assert res2.row_loss - ce == pytest.approx(-np.log(p[np.arange(4), cls]), rel=1e-12)
+
+
+@pytest.mark.parametrize("T", [1.0, 2.5])
+def test_kl_directions_swap_and_average(T):
+    """The reverse direction with own and peer exchanged is the forward direction (same number), and the
+    symmetric form is the average of the two; the reverse gradient is T p ((log p - log t) - KL(p || t))."""
+    own, peers, labels = rng_inputs(31, 6, 11, 2)
+    kw = dict(alpha=1.0, temperature=T, reduction=oracle.REDUCE_SUM)
+    ce_own = oracle.codistill(own, [], labels, reduction=oracle.REDUCE_SUM).row_loss
+    ce_peer = oracle.codistill(peers[0], [], labels, reduction=oracle.REDUCE_SUM).row_loss
+    fwd = oracle.codistill(own, peers, labels, dist=oracle.DIST_KL, **kw)
+    rev = oracle.codistill(own, peers, labels, dist=oracle.DIST_KL_REVERSE, **kw)
+    sym = oracle.codistill(own, peers, labels, dist=oracle.DIST_KL_SYMMETRIC, **kw)
+    fwd_swapped = oracle.codistill(peers[0], [own], labels, dist=oracle.DIST_KL, **kw)
+    assert rev.row_loss - ce_own == pytest.approx(fwd_swapped.row_loss - ce_peer, rel=1e-12, abs=1e-14)
+    assert sym.row_loss == pytest.approx(0.5 * (fwd.row_loss + rev.row_loss), rel=1e-13)
+    assert sym.grad == pytest.approx(0.5 * (fwd.grad + rev.grad), abs=1e-14)
+    # the closed form of the reverse gradient, written out with numpy
+    z, v = widen(own) / T, widen(peers[0]) / T
+    lp = z - np.log(np.exp(z - z.max(1, keepdims=True)).sum(1, keepdims=True)) - z.max(1, keepdims=True)
+    lt = v - np.log(np.exp(v - v.max(1, keepdims=True)).sum(1, keepdims=True)) - v.max(1, keepdims=True)
+    p = np.exp(lp)
+    kl = (p * (lp - lt)).sum(1, keepdims=True)
+    ce_grad = oracle.codistill(own, [], labels, reduction=oracle.REDUCE_SUM).grad
+    assert rev.grad - ce_grad == pytest.approx(T * p * ((lp - lt) - kl), abs=1e-13)
+    assert rev.row_loss - ce_own == pytest.approx(T * T * kl[:, 0], rel=1e-12)
+    assert np.all(rev.row_loss - ce_own >= 0) and np.all(fwd.row_loss - ce_own >= 0)    # a divergence is never negative
 
 
 def test_kl_temperature_scaling():
@@ -331,8 +359,10 @@ def _torch_reference(own, peers, labels, mask, alpha, T, eps, dist, pr, red):
             elif dist == oracle.DIST_MSE_CENTRED:
                 ds.append(F.mse_loss(z - z.mean(1, keepdim=True), p - p.mean(1, keepdim=True), reduction="none").mean(1))
             else:
-                ds.append(T * T * F.kl_div(F.log_softmax(z / T, 1), F.log_softmax(p / T, 1), reduction="none",
-                                           log_target=True).sum(1))
+                lp, lt = F.log_softmax(z / T, 1), F.log_softmax(p / T, 1)
+                fwd = T * T * F.kl_div(lp, lt, reduction="none", log_target=True).sum(1)    # KL(t || p)
+                rev = T * T * F.kl_div(lt, lp, reduction="none", log_target=True).sum(1)    # KL(p || t)
+                ds.append({oracle.DIST_KL: fwd, oracle.DIST_KL_REVERSE: rev, oracle.DIST_KL_SYMMETRIC: 0.5 * (fwd + rev)}[dist])
         row = ce + alpha * torch.stack(ds).mean(0)
     else:
         row = ce
