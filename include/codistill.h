@@ -60,8 +60,11 @@ enum { CODISTILL_F32 = 0, CODISTILL_BF16 = 1 };
 enum {
   CODISTILL_DIST_MSE_LOGITS = 0, /* D(z, z') = 1/C * sum_c (z_c - z'_c)^2 (Appendix "Implementation Details") */
   CODISTILL_DIST_KL_SOFTMAX = 1, /* D(z, z') = T^2 * KL(softmax(z'/T) || softmax(z/T)) (Section 2, earlier work) */
-  CODISTILL_DIST_MSE_CENTRED = 2 /* MSE between logits centred on their class means (Appendix "Implementation Details":
+  CODISTILL_DIST_MSE_CENTRED = 2, /* MSE between logits centred on their class means (Appendix "Implementation Details":
                                     centring gave similar results): D(z, z') = 1/C * sum_c ((z_c - mean z) - (z'_c - mean z'))^2 */
+  CODISTILL_DIST_KL_REVERSE = 3, /* the other direction of Section 2's KL divergence (the paper does not fix it):
+                                    D(z, z') = T^2 * KL(softmax(z/T) || softmax(z'/T)) */
+  CODISTILL_DIST_KL_SYMMETRIC = 4 /* half the sum of the two directions */
 };
 
 /* how the n-1 peers enter D */
@@ -262,6 +265,21 @@ size_t codistill_all_workspace_bytes(int n, int64_t rows);
 
 /* Human-readable name of a CODISTILL_ERR_* code (static storage). */
 const char* codistill_status_string(int status);
+
+/*
+ * Compression of the predictions exchanged between the model groups (Section 3: every device sends the
+ * predictions of its minibatch, b_pred bits per sample, to the devices that train the other models).
+ * Packing 32-bit logits to bfloat16 (round to nearest, ties to even; NaN stays NaN) halves b_pred; the
+ * receiver either runs the loss on the bfloat16 tensors or widens them again (exact) with the second call.
+ *   src / dst      DEVICE pointers, row-major [rows, stride] with stride >= classes (elements); only the first
+ *                  `classes` elements of a row are read and written.  16-byte aligned bases with pitches that
+ *                  are multiples of 8 (bf16) / 4 (fp32) elements take the 16-byte path, anything else works too.
+ * Asynchronous on `stream`; CODISTILL_ERR_SHAPE / CODISTILL_ERR_NULL on bad arguments, nothing launched.
+ */
+int codistill_pack_predictions(const float* src, void* dst_bf16, int64_t rows, int64_t classes, int64_t src_stride,
+                               int64_t dst_stride, void* stream);
+int codistill_unpack_predictions(const void* src_bf16, float* dst, int64_t rows, int64_t classes, int64_t src_stride,
+                                 int64_t dst_stride, void* stream);
 
 /*
  * Diagnostic, not part of the objective.  Every wait of the kernels on an asynchronous copy is bounded:

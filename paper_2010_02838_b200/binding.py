@@ -17,7 +17,7 @@ LIB_PATH = os.path.join(_HERE, "libcodistill.so")
 
 OK = 0
 F32, BF16 = 0, 1
-DIST_MSE_LOGITS, DIST_KL_SOFTMAX, DIST_MSE_CENTRED = 0, 1, 2
+DIST_MSE_LOGITS, DIST_KL_SOFTMAX, DIST_MSE_CENTRED, DIST_KL_REVERSE, DIST_KL_SYMMETRIC = 0, 1, 2, 3, 4
 PEERS_PAIRWISE_MEAN, PEERS_MEAN_TARGET = 0, 1
 REDUCE_MEAN_VALID, REDUCE_SUM = 0, 1
 DEV_BAD_LABEL, DEV_TIMEOUT = 1, 2
@@ -31,7 +31,7 @@ EXPORTS = (
     "codistill_loss_fwd_bwd_static", "codistill_loss_fwd_bwd_all", "codistill_all_workspace_bytes",
     "codistill_workspace_bytes", "codistill_host_workspace_bytes", "codistill_status_string",
     "codistill_version", "codistill_kernel_regime", "codistill_last_cuda_error",
-    "codistill_selftest_bounded_wait",
+    "codistill_selftest_bounded_wait", "codistill_pack_predictions", "codistill_unpack_predictions",
     "codistill_schedule_alpha", "codistill_schedule_piecewise", "codistill_schedule_step_decay",
     "codistill_is_exchange_step", "codistill_bits_all_reduce", "codistill_bits_checkpoints",
     "codistill_bits_predictions",
@@ -135,6 +135,9 @@ def load_library() -> ctypes.CDLL:
     lib.codistill_host_workspace_bytes.argtypes = [i32, i64, i64, i32, i64]
     lib.codistill_status_string.restype = ctypes.c_char_p
     lib.codistill_status_string.argtypes = [i32]
+    for fn in (lib.codistill_pack_predictions, lib.codistill_unpack_predictions):
+        fn.restype = i32
+        fn.argtypes = [vp, vp, i64, i64, i64, i64, vp]
     lib.codistill_selftest_bounded_wait.restype = i32
     lib.codistill_selftest_bounded_wait.argtypes = [vp, ctypes.c_uint64, vp]
     lib.codistill_last_cuda_error.restype = ctypes.c_char_p
@@ -401,6 +404,46 @@ class AllPlan:
         if rc != OK:
             raise CodistillError(rc)
         return self.out
+
+
+def _rows_and_pitch(t: torch.Tensor):
+    if t.dim() != 2 or t.stride(1) != 1:
+        raise ValueError("predictions must be [rows, classes] with unit inner stride")
+    return t.shape[0], t.shape[1], (t.stride(0) if t.shape[0] > 1 else max(t.stride(0), t.shape[1]))
+
+
+def pack_predictions(logits: torch.Tensor, out: torch.Tensor | None = None, stream: torch.cuda.Stream | None = None) -> torch.Tensor:
+    """fp32 predictions -> bfloat16 (round to nearest even) on the device, for the exchange between model groups."""
+    _require_cuda(logits, out)
+    if logits.dtype != torch.float32:
+        raise TypeError("pack_predictions takes float32 logits")
+    rows, C, pitch = _rows_and_pitch(logits)
+    if out is None:
+        out = torch.empty((rows, C), dtype=torch.bfloat16, device=logits.device)
+    orows, oC, opitch = _rows_and_pitch(out)
+    if (orows, oC) != (rows, C) or out.dtype != torch.bfloat16:
+        raise ValueError("out must be a bfloat16 tensor of the same shape")
+    rc = load_library().codistill_pack_predictions(_ptr(logits), _ptr(out), rows, C, pitch, opitch, _stream_ptr(stream))
+    if rc != OK:
+        raise CodistillError(rc)
+    return out
+
+
+def unpack_predictions(packed: torch.Tensor, out: torch.Tensor | None = None, stream: torch.cuda.Stream | None = None) -> torch.Tensor:
+    """bfloat16 predictions -> fp32 (exact) on the device."""
+    _require_cuda(packed, out)
+    if packed.dtype != torch.bfloat16:
+        raise TypeError("unpack_predictions takes bfloat16 predictions")
+    rows, C, pitch = _rows_and_pitch(packed)
+    if out is None:
+        out = torch.empty((rows, C), dtype=torch.float32, device=packed.device)
+    orows, oC, opitch = _rows_and_pitch(out)
+    if (orows, oC) != (rows, C) or out.dtype != torch.float32:
+        raise ValueError("out must be a float32 tensor of the same shape")
+    rc = load_library().codistill_unpack_predictions(_ptr(packed), _ptr(out), rows, C, pitch, opitch, _stream_ptr(stream))
+    if rc != OK:
+        raise CodistillError(rc)
+    return out
 
 
 def selftest_bounded_wait(limit_ns: int = 1_000_000, stream: torch.cuda.Stream | None = None) -> torch.Tensor:

@@ -10,7 +10,7 @@ _HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(_HERE, "csrc")
 OBJ_DIR = os.path.join(_HERE, "_build")
 LIB = os.path.join(_HERE, "libcodistill.so")
-SOURCES = ["api.cu", "rows_generic.cu", "rows_tma.cu", "rows_stream.cu", "rows_stream_kl.cu", "rows_all.cu", "rows_cluster.cu", "schedule.cu"]
+SOURCES = ["api.cu", "rows_generic.cu", "rows_tma.cu", "rows_stream.cu", "rows_stream_kl.cu", "rows_all.cu", "rows_cluster.cu", "schedule.cu", "predictions.cu"]
 HEADERS = ["common.cuh", "seg_math.cuh", "stream_common.cuh", "bulk_copy.cuh", "cluster_args.cuh", os.path.join("..", "..", "include", "codistill.h"),
            os.path.join("..", "..", "include", "codistill_schedule.h")]
 NVCC_FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",

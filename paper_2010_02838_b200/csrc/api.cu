@@ -135,8 +135,7 @@ static int validate(const codistill_params_t* p, bool host_pointers) {
   if (p->dtype != CODISTILL_F32 && p->dtype != CODISTILL_BF16) return CODISTILL_ERR_DTYPE;
   if (!(p->temperature > 0.f) || !isfinite(p->temperature) || !isfinite(p->alpha)) return CODISTILL_ERR_PARAM;
   if (!(p->label_smoothing >= 0.f && p->label_smoothing < 1.f)) return CODISTILL_ERR_PARAM;
-  if (p->dist_kind != CODISTILL_DIST_MSE_LOGITS && p->dist_kind != CODISTILL_DIST_KL_SOFTMAX &&
-      p->dist_kind != CODISTILL_DIST_MSE_CENTRED) return CODISTILL_ERR_PARAM;
+  if (p->dist_kind < CODISTILL_DIST_MSE_LOGITS || p->dist_kind > CODISTILL_DIST_KL_SYMMETRIC) return CODISTILL_ERR_PARAM;
   if (p->peer_reduce != CODISTILL_PEERS_PAIRWISE_MEAN && p->peer_reduce != CODISTILL_PEERS_MEAN_TARGET) return CODISTILL_ERR_PARAM;
   if (p->reduction != CODISTILL_REDUCE_MEAN_VALID && p->reduction != CODISTILL_REDUCE_SUM) return CODISTILL_ERR_PARAM;
   if (p->n - 1 > kMaxPeers) return CODISTILL_ERR_UNSUPPORTED;

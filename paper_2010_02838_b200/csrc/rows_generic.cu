@@ -12,9 +12,10 @@ namespace codistill {
 constexpr int kWarpRegimeThreads = 256;   // 8 rows per CTA
 constexpr int kBlockRegimeThreads = 512;
 
-struct PeerStats {       // per-peer row statistics kept in shared memory (KL form)
+struct PeerStats {       // per-peer row statistics kept in shared memory (KL forms)
   float max_v[kMaxPeers];
   float log_sum[kMaxPeers];
+  float kl_rev[kMaxPeers];   // KL(p^T || t_j), the row constant in the reverse direction's gradient
 };
 
 template <typename T, int V, int G>
@@ -41,7 +42,10 @@ __device__ __forceinline__ void process_row(const KArgs& a, int64_t r, int lane,
     return;
   }
   const int y = a.labels[r];
-  const bool kl = (a.dist == CODISTILL_DIST_KL_SOFTMAX);
+  // the softmax-KL family: peer as target (forward), own as target (reverse), or half of each (symmetric)
+  const bool kl = a.dist == CODISTILL_DIST_KL_SOFTMAX || a.dist == CODISTILL_DIST_KL_REVERSE || a.dist == CODISTILL_DIST_KL_SYMMETRIC;
+  const float wf = a.dist == CODISTILL_DIST_KL_SOFTMAX ? 1.f : a.dist == CODISTILL_DIST_KL_SYMMETRIC ? 0.5f : 0.f;
+  const float wr = a.dist == CODISTILL_DIST_KL_REVERSE ? 1.f : a.dist == CODISTILL_DIST_KL_SYMMETRIC ? 0.5f : 0.f;
   const bool centred = (a.dist == CODISTILL_DIST_MSE_CENTRED);  // MSE between logits centred on their class means
   const bool with_term = (P >= 1 && a.alpha != 0.f);
   const float inv_T = 1.f / a.temperature;
@@ -125,7 +129,25 @@ __device__ __forceinline__ void process_row(const KArgs& a, int64_t r, int lane,
             if (k * V + i < C) sj[0] += expf((v[i] - pb) * inv_T);
         }
         Group<G>::sum(sj, scratch);
-        if (lane == 0) { ps->max_v[j] = pb; ps->log_sum[j] = logf(sj[0]); }
+        const float lsj = logf(sj[0]);
+        if (lane == 0) { ps->max_v[j] = pb; ps->log_sum[j] = lsj; }
+        if (wr != 0.f) {   // KL(p^T || t_j) = sum_c p^T_c (log p^T_c - log t_jc)
+          float kj[1] = {0.f};
+          for (int64_t k = lane; k < n_packets; k += G) {
+            float v[V], o[V];
+            load_packet<T, V>(p_row, k * V, v);
+            load_packet<T, V>(z_row, k * V, o);
+#pragma unroll
+            for (int i = 0; i < V; ++i) {
+              if (k * V + i < C) {
+                const float log_p = (o[i] - m) * inv_T - log_ST, log_t = (v[i] - pb) * inv_T - lsj;
+                kj[0] = fmaf(expf(log_p), log_p - log_t, kj[0]);
+              }
+            }
+          }
+          Group<G>::sum(kj, scratch);
+          if (lane == 0) ps->kl_rev[j] = kj[0];
+        }
       }
     }
     if (peer_stats || peer_means) {
@@ -134,7 +156,7 @@ __device__ __forceinline__ void process_row(const KArgs& a, int64_t r, int lane,
   }
 
   // ---- KL against the averaged peer: statistics of zbar / T
-  float mb = 0.f, log_Sb = 0.f;
+  float mb = 0.f, log_Sb = 0.f, kl_rev_b = 0.f;
   const float inv_P = P >= 1 ? 1.f / (float)P : 0.f;
   if (with_term && kl && a.peer_reduce == CODISTILL_PEERS_MEAN_TARGET) {
     float bm = -INFINITY;
@@ -170,6 +192,30 @@ __device__ __forceinline__ void process_row(const KArgs& a, int64_t r, int lane,
     }
     Group<G>::sum(sb, scratch);
     log_Sb = logf(sb[0]);
+    if (wr != 0.f) {   // KL(p^T || t) against the softmax of the averaged peers
+      float kb[1] = {0.f};
+      for (int64_t k = lane; k < n_packets; k += G) {
+        float zb[V], o[V];
+#pragma unroll
+        for (int i = 0; i < V; ++i) zb[i] = 0.f;
+        for (int j = 0; j < P; ++j) {
+          float v[V];
+          load_packet<T, V>(reinterpret_cast<const T*>(a.peers[j]) + lr * a.row_stride, k * V, v);
+#pragma unroll
+          for (int i = 0; i < V; ++i) zb[i] += v[i];
+        }
+        load_packet<T, V>(z_row, k * V, o);
+#pragma unroll
+        for (int i = 0; i < V; ++i) {
+          if (k * V + i < C) {
+            const float log_p = (o[i] - m) * inv_T - log_ST, log_t = (zb[i] * inv_P - mb) * inv_T - log_Sb;
+            kb[0] = fmaf(expf(log_p), log_p - log_t, kb[0]);
+          }
+        }
+      }
+      Group<G>::sum(kb, scratch);
+      kl_rev_b = kb[0];
+    }
   }
 
   // ---- element-wise pass: distillation term and gradient
@@ -222,17 +268,19 @@ __device__ __forceinline__ void process_row(const KArgs& a, int64_t r, int lane,
             for (int j = 0; j < P; ++j) {
               float u[V];
               load_packet<T, V>(reinterpret_cast<const T*>(a.peers[j]) + lr * a.row_stride, c0, u);
-              const float mj = ps->max_v[j], lsj = ps->log_sum[j];
+              const float mj = ps->max_v[j], lsj = ps->log_sum[j], kj = ps->kl_rev[j];
 #pragma unroll
               for (int i = 0; i < V; ++i) {
                 const float log_t = (u[i] - mj) * inv_T - lsj;
                 const float t = expf(log_t);
-                tbar[i] += t;
-                if (c0 + i < C) dacc[0] = fmaf(t, log_t - log_pT[i], dacc[0]);
+                const float diff = log_pT[i] - log_t;
+                // forward: t (log t - log p), derivative T (p - t); reverse: p (log p - log t), derivative T p (diff - KL_j)
+                tbar[i] += wf * (pT[i] - t) + wr * pT[i] * (diff - kj);
+                if (c0 + i < C) dacc[0] += wr * pT[i] * diff - wf * t * diff;
               }
             }
 #pragma unroll
-            for (int i = 0; i < V; ++i) dD[i] = temp * (pT[i] - tbar[i] * inv_P);
+            for (int i = 0; i < V; ++i) dD[i] = temp * tbar[i] * inv_P;
           } else {
             float zb[V];
 #pragma unroll
@@ -247,8 +295,9 @@ __device__ __forceinline__ void process_row(const KArgs& a, int64_t r, int lane,
             for (int i = 0; i < V; ++i) {
               const float log_t = (zb[i] * inv_P - mb) * inv_T - log_Sb;
               const float t = expf(log_t);
-              if (c0 + i < C) dacc[0] = fmaf(t, log_t - log_pT[i], dacc[0]);
-              dD[i] = temp * (pT[i] - t);
+              const float diff = log_pT[i] - log_t;
+              if (c0 + i < C) dacc[0] += wr * pT[i] * diff - wf * t * diff;
+              dD[i] = temp * (wf * (pT[i] - t) + wr * pT[i] * (diff - kl_rev_b));
             }
           }
         }

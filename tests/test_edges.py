@@ -25,7 +25,7 @@ def rand_inputs(seed, rows, C, n, dtype, scale=1.5):
 
 @pytest.mark.parametrize("dtype", ["f32", "bf16"])
 @pytest.mark.parametrize("C", [1, 2, 7, 33, 257, 1000, 1023, 4099, 9001, 20011])
-@pytest.mark.parametrize("dist", [0, 1, 2])
+@pytest.mark.parametrize("dist", [0, 1, 2, 3, 4])
 def test_ragged_class_counts(dtype, C, dist):
     rows = 37 if C < 5000 else 11
     own, peers, labels = rand_inputs(C, rows, C, 3, dtype)

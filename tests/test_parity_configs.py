@@ -13,7 +13,7 @@ from helpers import compare
 
 pytestmark = pytest.mark.gpu
 
-DISTS = [cb.DIST_MSE_LOGITS, cb.DIST_KL_SOFTMAX, cb.DIST_MSE_CENTRED]
+DISTS = [cb.DIST_MSE_LOGITS, cb.DIST_KL_SOFTMAX, cb.DIST_MSE_CENTRED, cb.DIST_KL_REVERSE, cb.DIST_KL_SYMMETRIC]
 PEERS = [cb.PEERS_PAIRWISE_MEAN, cb.PEERS_MEAN_TARGET]
 REDS = [cb.REDUCE_SUM, cb.REDUCE_MEAN_VALID]
 
