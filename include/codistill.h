@@ -303,14 +303,15 @@ int codistill_version(void);
 
 /*
  * Name of the kernel regime the dispatcher picks for a problem, so that tests and benchmarks can
- * state which kernel they exercised: "warp" (rows up to 8 KiB, one warp per row), "tma" (long rows,
+ * state which kernel they exercised: "short" (up to 1024 classes, up to 7 peers, MSE distance, at most 16384
+ * rows: one launch, one warp per row, the row held in registers), "warp" (rows up to 8 KiB, one warp per row), "tma" (long rows,
  * MSE distance, own row staged in shared memory by bulk copies), "stream" (long rows, direct loads,
  * own row read twice: MSE rows beyond 64 KiB, the softmax-KL and centred-MSE distances), "cluster"
  * (long rows, all n row images of a row index kept in the shared memory of a thread-block cluster: by
  * default only the peer counts the two kernels before are not built for, 4 to 6) or "block"
  * (everything else).  The answer assumes
  * 16-byte aligned tensor bases (the long-row kernels need them).  For measurements the environment
- * variable CODISTILL_REGIME = tma | stream | cluster | block overrides the choice where the named
+ * variable CODISTILL_REGIME = warp | tma | stream | cluster | block overrides the choice where the named
  * kernel can serve the call, and CODISTILL_CLUSTER_SIZE = 1 | 2 | 4 | 8 | 16 fixes the number of
  * CTAs per cluster of the "cluster" kernel.  Static storage; NULL on bad arguments.
  */

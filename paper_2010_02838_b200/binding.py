@@ -407,7 +407,7 @@ class AllPlan:
 
 
 def _rows_and_pitch(t: torch.Tensor):
-    if t.dim() != 2 or t.stride(1) != 1:
+    if t.dim() != 2 or (t.numel() > 0 and t.shape[1] > 1 and t.stride(1) != 1):
         raise ValueError("predictions must be [rows, classes] with unit inner stride")
     return t.shape[0], t.shape[1], (t.stride(0) if t.shape[0] > 1 else max(t.stride(0), t.shape[1]))
 

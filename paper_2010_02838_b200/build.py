@@ -10,7 +10,7 @@ _HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(_HERE, "csrc")
 OBJ_DIR = os.path.join(_HERE, "_build")
 LIB = os.path.join(_HERE, "libcodistill.so")
-SOURCES = ["api.cu", "rows_generic.cu", "rows_tma.cu", "rows_stream.cu", "rows_stream_kl.cu", "rows_all.cu", "rows_cluster.cu", "schedule.cu", "predictions.cu"]
+SOURCES = ["api.cu", "rows_generic.cu", "rows_tma.cu", "rows_stream.cu", "rows_stream_kl.cu", "rows_all.cu", "rows_cluster.cu", "schedule.cu", "predictions.cu", "rows_short.cu"]
 HEADERS = ["common.cuh", "seg_math.cuh", "stream_common.cuh", "bulk_copy.cuh", "cluster_args.cuh", os.path.join("..", "..", "include", "codistill.h"),
            os.path.join("..", "..", "include", "codistill_schedule.h")]
 NVCC_FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
@@ -25,9 +25,17 @@ def _stale() -> bool:
     return any(os.path.getmtime(d) > t for d in deps)
 
 
-def _compile(nvcc: str, src: str):
+def _compile(nvcc: str, src: str, force: bool):
+    """One object per source; an object newer than its source, every header and this script is kept."""
     obj = os.path.join(OBJ_DIR, os.path.splitext(src)[0] + ".o")
+    log = obj + ".log"
+    deps = [os.path.join(CSRC, src)] + [os.path.join(CSRC, h) for h in HEADERS] + [os.path.abspath(__file__)]
+    if not force and os.path.exists(obj) and os.path.exists(log) and all(os.path.getmtime(d) <= os.path.getmtime(obj) for d in deps):
+        return obj, subprocess.CompletedProcess([], 0, open(log).read(), "")
     res = subprocess.run([nvcc, *NVCC_FLAGS, "-c", "-o", obj, os.path.join(CSRC, src)], capture_output=True, text=True)
+    if res.returncode == 0:
+        with open(log, "w") as f:
+            f.write(res.stdout + res.stderr)
     return obj, res
 
 
@@ -38,7 +46,7 @@ def build(force: bool = False, verbose: bool = False) -> str:
         nvcc = os.environ.get("NVCC", "/usr/local/cuda/bin/nvcc")
         os.makedirs(OBJ_DIR, exist_ok=True)
         with ThreadPoolExecutor(max_workers=min(len(SOURCES), os.cpu_count() or 1)) as pool:
-            results = list(pool.map(lambda s: _compile(nvcc, s), SOURCES))
+            results = list(pool.map(lambda s: _compile(nvcc, s, force), SOURCES))
         log = "".join(r.stdout + r.stderr for _, r in results)
         failed = [r for _, r in results if r.returncode != 0]
         if verbose or failed:

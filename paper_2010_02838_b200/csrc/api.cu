@@ -21,6 +21,8 @@ int tma_ctas_per_sm(const KArgs& a, int dtype, int smem_optin);
 cudaError_t launch_tma(const KArgs& a, int dtype, int num_sms, int smem_optin, cudaStream_t stream);
 bool stream_supported(const KArgs& a, int dtype);
 cudaError_t launch_stream(const KArgs& a, int dtype, int num_sms, cudaStream_t stream);
+bool short_supported(const KArgs& a, int dtype);
+cudaError_t launch_short(const KArgs& a, int dtype, bool vec, int num_sms, cudaStream_t stream);
 bool cluster_supported(const KArgs& a, int dtype, int smem_optin);
 cudaError_t launch_cluster_single(const KArgs& a, int dtype, int smem_optin, cudaStream_t stream);
 
@@ -178,6 +180,12 @@ static Regime pick_regime(const KArgs& a, int dtype, int smem_optin) {
   return generic;
 }
 
+// CODISTILL_REGIME=warp (or block) keeps short rows on the two-launch generic kernels, for measurements
+static bool regime_forced_away_from_short() {
+  const char* want = getenv("CODISTILL_REGIME");
+  return want != nullptr && (strcmp(want, "warp") == 0 || strcmp(want, "block") == 0);
+}
+
 static bool rows_vectorizable(const KArgs& a, int dtype) {
   const size_t es = dtype == CODISTILL_F32 ? 4 : 2;
   if ((a.row_stride * es) % 16 != 0) return false;
@@ -257,6 +265,9 @@ static int run_device(const codistill_params_t* p, cudaStream_t stream) {
   if (const int rc_cuda = cuda_status(device_info(&di))) return rc_cuda;
   KArgs a;
   fill_args(&a, p, p->workspace);
+  // short rows: one cooperative launch does the counting, the rows and the final reduction
+  if (short_supported(a, p->dtype) && !regime_forced_away_from_short())
+    return cuda_status(launch_short(a, p->dtype, rows_vectorizable(a, p->dtype), di.num_sms, stream));
   if (const int rc_cuda = cuda_status(launch_prep(a, stream))) return rc_cuda;
   if (p->rows == 0) {
     a.fused_finalize = 0;
@@ -513,6 +524,8 @@ const char* codistill_kernel_regime(int n, int64_t rows, int64_t classes, int64_
   a.peer_reduce = peer_reduce;
   a.row_end = rows;
   a.rows_total = rows;
+  a.fused_finalize = 1;
+  if (short_supported(a, dtype) && !regime_forced_away_from_short()) return "short";
   switch (pick_regime(a, dtype, di.smem_optin)) {
     case kRegimeWarp: return "warp";
     case kRegimeBlock: return "block";

@@ -140,8 +140,10 @@ __device__ __forceinline__ void process_row(const KArgs& a, int64_t r, int lane,
 #pragma unroll
             for (int i = 0; i < V; ++i) {
               if (k * V + i < C) {
-                const float log_p = (o[i] - m) * inv_T - log_ST, log_t = (v[i] - pb) * inv_T - lsj;
-                kj[0] = fmaf(expf(log_p), log_p - log_t, kj[0]);
+                // log p - log t with the large parts cancelled before they are rounded
+                const float log_p = (o[i] - m) * inv_T - log_ST;
+                const float diff = ((o[i] - v[i]) - (m - pb)) * inv_T - (log_ST - lsj);
+                kj[0] = fmaf(expf(log_p), diff, kj[0]);
               }
             }
           }
@@ -208,8 +210,9 @@ __device__ __forceinline__ void process_row(const KArgs& a, int64_t r, int lane,
 #pragma unroll
         for (int i = 0; i < V; ++i) {
           if (k * V + i < C) {
-            const float log_p = (o[i] - m) * inv_T - log_ST, log_t = (zb[i] * inv_P - mb) * inv_T - log_Sb;
-            kb[0] = fmaf(expf(log_p), log_p - log_t, kb[0]);
+            const float log_p = (o[i] - m) * inv_T - log_ST;
+            const float diff = ((o[i] - zb[i] * inv_P) - (m - mb)) * inv_T - (log_ST - log_Sb);
+            kb[0] = fmaf(expf(log_p), diff, kb[0]);
           }
         }
       }
@@ -268,12 +271,12 @@ __device__ __forceinline__ void process_row(const KArgs& a, int64_t r, int lane,
             for (int j = 0; j < P; ++j) {
               float u[V];
               load_packet<T, V>(reinterpret_cast<const T*>(a.peers[j]) + lr * a.row_stride, c0, u);
-              const float mj = ps->max_v[j], lsj = ps->log_sum[j], kj = ps->kl_rev[j];
+              const float mj = ps->max_v[j], lsj = ps->log_sum[j], kj = wr != 0.f ? ps->kl_rev[j] : 0.f;   // unset without a reverse part
 #pragma unroll
               for (int i = 0; i < V; ++i) {
                 const float log_t = (u[i] - mj) * inv_T - lsj;
                 const float t = expf(log_t);
-                const float diff = log_pT[i] - log_t;
+                const float diff = ((v[i] - u[i]) - (m - mj)) * inv_T - (log_ST - lsj);   // log p - log t, large parts cancelled first
                 // forward: t (log t - log p), derivative T (p - t); reverse: p (log p - log t), derivative T p (diff - KL_j)
                 tbar[i] += wf * (pT[i] - t) + wr * pT[i] * (diff - kj);
                 if (c0 + i < C) dacc[0] += wr * pT[i] * diff - wf * t * diff;
@@ -295,7 +298,7 @@ __device__ __forceinline__ void process_row(const KArgs& a, int64_t r, int lane,
             for (int i = 0; i < V; ++i) {
               const float log_t = (zb[i] * inv_P - mb) * inv_T - log_Sb;
               const float t = expf(log_t);
-              const float diff = log_pT[i] - log_t;
+              const float diff = ((v[i] - zb[i] * inv_P) - (m - mb)) * inv_T - (log_ST - log_Sb);
               if (c0 + i < C) dacc[0] += wr * pT[i] * diff - wf * t * diff;
               dD[i] = temp * (wf * (pT[i] - t) + wr * pT[i] * (diff - kl_rev_b));
             }

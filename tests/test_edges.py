@@ -194,3 +194,31 @@ def test_expired_wait_sets_the_status_bit_and_the_context_stays_usable():
     compare(own, peers, labels, None, alpha=1.0, reduction=cb.REDUCE_SUM, expect_regime="tma")
     with pytest.raises(cb.CodistillError):
         cb.selftest_bounded_wait(10 ** 9)     # limits beyond 100 ms are refused on the host
+
+
+@pytest.mark.parametrize("dtype", ["f32", "bf16"])
+@pytest.mark.parametrize("C,n", [(1, 2), (10, 2), (33, 4), (257, 8), (1000, 3), (1024, 8), (1023, 1)])
+def test_single_launch_short_row_kernel(dtype, C, n):
+    """Short rows in one cooperative launch: every lane count per row, ragged last packets, a mask with a bad
+    label, planted arg-max ties, both reductions, guard bands around the gradient, two identical runs."""
+    rows = 77
+    own, peers, labels = rand_inputs(5 * C + n, rows, C, n, dtype, scale=2.0)
+    mask = (np.arange(rows) % 6 != 4).astype(np.uint8)
+    labels[3] = C + 5                      # a label that is not a class: the row counts as masked, status bit raised
+    if C > 4:
+        for r in range(0, rows, 5):        # equal maxima in own and peers: the first one decides
+            own[r, [1, C - 2]] = own[r].max() + 1
+            for p in peers:
+                p[r, [C - 2]] = p[r].max() + 1
+    for pr, red in ((cb.PEERS_PAIRWISE_MEAN, cb.REDUCE_SUM), (cb.PEERS_MEAN_TARGET, cb.REDUCE_MEAN_VALID)):
+        plan, out, ref = compare(own, peers, labels, mask, alpha=0.8, label_smoothing=0.1, peer_reduce=pr, reduction=red,
+                                 expect_regime="short")
+        assert int(out.status.item()) == cb.DEV_BAD_LABEL
+    g = torch.full((rows * C + 64,), 3.0, dtype=plan.out.grad.dtype, device="cuda")
+    plan.params.grad_logits = g[32:].data_ptr()
+    first = (out.grad.clone(), out.row_loss.clone(), out.loss.clone(), out.counters.clone())
+    plan.run()
+    torch.cuda.synchronize()
+    assert torch.all(g[:32].float() == 3.0) and torch.all(g[32 + rows * C:].float() == 3.0)
+    assert torch.equal(g[32:32 + rows * C].view(rows, C), first[0])
+    assert torch.equal(first[1], out.row_loss) and torch.equal(first[2], out.loss) and torch.equal(first[3], out.counters)

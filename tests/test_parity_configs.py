@@ -35,7 +35,7 @@ def test_workload_parity(idx, dist, pr, red):
     plan, _, _ = compare(own, peers, labels, mask, alpha=w.alpha, temperature=w.temperature,
                          label_smoothing=w.label_smoothing, dist=dist, peer_reduce=pr, reduction=red)
     if dist == cb.DIST_MSE_LOGITS:   # which kernel served the workload
-        assert plan.regime == {1: "warp", 2: "warp", 3: "warp", 4: "tma", 5: "stream"}[idx]
+        assert plan.regime == {1: "short", 2: "short", 3: "short", 4: "tma", 5: "stream"}[idx]
 
 
 @pytest.mark.parametrize("idx,regime", [(4, "stream"), (5, "tma")])
@@ -47,6 +47,18 @@ def test_workload_parity_other_long_row_kernel(monkeypatch, idx, regime, pr, red
     own, peers, labels, mask = synth.make_inputs(w)
     compare(own, peers, labels, mask, alpha=w.alpha, temperature=w.temperature, label_smoothing=w.label_smoothing,
             dist=cb.DIST_MSE_LOGITS, peer_reduce=pr, reduction=red, expect_regime=regime)
+
+
+@pytest.mark.parametrize("idx", [1, 2, 3])
+@pytest.mark.parametrize("pr,red", list(itertools.product(PEERS, REDS)))
+def test_short_workloads_on_the_two_launch_kernel(monkeypatch, idx, pr, red):
+    """The three small workloads on the warp-per-row kernel behind a counting launch (their default is the
+    single-launch kernel)."""
+    monkeypatch.setenv("CODISTILL_REGIME", "warp")
+    w = workload(idx)
+    own, peers, labels, mask = synth.make_inputs(w)
+    compare(own, peers, labels, mask, alpha=w.alpha, temperature=w.temperature, label_smoothing=w.label_smoothing,
+            dist=cb.DIST_MSE_LOGITS, peer_reduce=pr, reduction=red, expect_regime="warp")
 
 
 @pytest.mark.parametrize("idx", [1, 2, 3])
