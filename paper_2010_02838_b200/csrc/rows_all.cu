@@ -110,6 +110,7 @@ __global__ void __launch_bounds__(all_threads(N), all_ctas_per_sm(N)) rows_all_k
     w = 1.f / (float)(nv > 1 ? nv : 1);
   }
   const float inv_C = 1.f / (float)C;
+  const bool need_z = a.eps != 0.f || a.centred != 0;
   constexpr float kRatio = (float)N / (float)(N - 1);           // z_i - zbar_(-i) = kRatio * z'_i
   const float cd = with_term ? w * a.alpha * (2.f * inv_C) * kRatio : 0.f;  // z'_i -> w alpha dD_i/dz_i
   const float cq = w * a.eps * inv_C;
@@ -225,9 +226,10 @@ __global__ void __launch_bounds__(all_threads(N), all_ctas_per_sm(N)) rows_all_k
           float2 z2[H];
           SegOps<T>::unpack2(rw[i], z2);
 #pragma unroll
-          for (int h = 0; h < H; ++h) {
-            acc = __fadd2_rn(acc, exp_shift2<T>(z2[h], best[i], make_float2(kLog2e, kLog2e), make_float2(nm, nm)));
-            zs2[i] = __fadd2_rn(zs2[i], z2[h]);
+          for (int h = 0; h < H; ++h) acc = __fadd2_rn(acc, exp_shift2<T>(z2[h], best[i], make_float2(kLog2e, kLog2e), make_float2(nm, nm)));
+          if (need_z) {   // the sum of the logits: label smoothing and the centred distance only
+#pragma unroll
+            for (int h = 0; h < H; ++h) zs2[i] = __fadd2_rn(zs2[i], z2[h]);
           }
           s2[i] = acc;
         }
@@ -295,7 +297,7 @@ __global__ void __launch_bounds__(all_threads(N), all_ctas_per_sm(N)) rows_all_k
       a_own[i] = first_equal_global<T>(z_row[i], m_seg, g.head, C, m);
       mi[i] = m;
       cpi[i] = w * __frcp_rn(S);
-      cmi[i] = a.centred ? sum_z * inv_C : 0.f;
+      cmi[i] = sum_z * inv_C;   // class mean; turned into (average class mean) - (class mean) below
       if constexpr (KL) {
         float S_T = S;
         if (!t_one) {
@@ -313,8 +315,17 @@ __global__ void __launch_bounds__(all_threads(N), all_ctas_per_sm(N)) rows_all_k
       }
     }
 
+    {
+      float avg = 0.f;
+#pragma unroll
+      for (int i = 0; i < N; ++i) avg += cmi[i];
+      avg *= (1.f / (float)N);
+#pragma unroll
+      for (int i = 0; i < N; ++i) cmi[i] = avg - cmi[i];
+    }
+
     // ================= pass B: centring, distance terms, gradients
-    float dist[N], qs = 0.f;   // qs: sum over the columns of sum_j z'_j^2 (pairwise form)
+    float dist[N];
 #pragma unroll
     for (int i = 0; i < N; ++i) dist[i] = 0.f;
     // one column: values zc[] of the n models; returns the gradient elements in gc[]
@@ -339,12 +350,17 @@ __global__ void __launch_bounds__(all_threads(N), all_ctas_per_sm(N)) rows_all_k
         }
         return;
       }
-      float zp[N], mu = 0.f, q = 0.f;
+      // z'_i = z_i - mean_j z_j; the centred distance adds cmi[i] = (average class mean) - (class mean of model i)
+      float zp[N], mu = zc[0];
 #pragma unroll
-      for (int i = 0; i < N; ++i) { zp[i] = zc[i] - cmi[i]; mu += zp[i]; }
-      mu *= (1.f / (float)N);
+      for (int i = 1; i < N; ++i) mu += zc[i];
+      mu *= (-1.f / (float)N);
 #pragma unroll
-      for (int i = 0; i < N; ++i) { zp[i] -= mu; q = fmaf(zp[i], zp[i], q); }
+      for (int i = 0; i < N; ++i) zp[i] = zc[i] + mu;
+      if (a.centred) {
+#pragma unroll
+        for (int i = 0; i < N; ++i) zp[i] += cmi[i];
+      }
       const float cqc = (c == (int64_t)y) ? cq + cy : cq;
 #pragma unroll
       for (int i = 0; i < N; ++i) {
@@ -353,9 +369,8 @@ __global__ void __launch_bounds__(all_threads(N), all_ctas_per_sm(N)) rows_all_k
         gc[i] = fmaf(e, cpi[i], fmaf(cd, zp[i], -cqc));
         dist[i] = fmaf(zp[i], zp[i], dist[i]);   // z'_i^2 = (z_i - zbar_(-i))^2 / kRatio^2; pairwise form: see the row results
       }
-      if constexpr (PW) qs += q;
     };
-    [[maybe_unused]] float2 dist2[N], qs2 = make_float2(0.f, 0.f);
+    [[maybe_unused]] float2 dist2[N];
 #pragma unroll
     for (int i = 0; i < N; ++i) dist2[i] = make_float2(0.f, 0.f);
     // two neighbouring columns c, c + 1 of the n models at once (packed fp32 pairs; bf16 logits)
@@ -389,12 +404,16 @@ __global__ void __launch_bounds__(all_threads(N), all_ctas_per_sm(N)) rows_all_k
         }
         return;
       }
-      float2 zp[N], mu = make_float2(0.f, 0.f), q = make_float2(0.f, 0.f);
+      float2 zp[N], mu = zc[0];
 #pragma unroll
-      for (int i = 0; i < N; ++i) { zp[i] = __fadd2_rn(zc[i], make_float2(-cmi[i], -cmi[i])); mu = __fadd2_rn(mu, zp[i]); }
+      for (int i = 1; i < N; ++i) mu = __fadd2_rn(mu, zc[i]);
       mu = __fmul2_rn(mu, make_float2(-1.f / (float)N, -1.f / (float)N));
 #pragma unroll
-      for (int i = 0; i < N; ++i) { zp[i] = __fadd2_rn(zp[i], mu); q = __ffma2_rn(zp[i], zp[i], q); }
+      for (int i = 0; i < N; ++i) zp[i] = __fadd2_rn(zc[i], mu);
+      if (a.centred) {
+#pragma unroll
+        for (int i = 0; i < N; ++i) zp[i] = __fadd2_rn(zp[i], make_float2(cmi[i], cmi[i]));
+      }
       const float2 ncq = make_float2((c == (int64_t)y) ? -(cq + cy) : -cq, (c + 1 == (int64_t)y) ? -(cq + cy) : -cq);
 #pragma unroll
       for (int i = 0; i < N; ++i) {
@@ -403,7 +422,6 @@ __global__ void __launch_bounds__(all_threads(N), all_ctas_per_sm(N)) rows_all_k
         gc[i] = __ffma2_rn(e, make_float2(cpi[i], cpi[i]), __ffma2_rn(make_float2(cd, cd), zp[i], ncq));
         dist2[i] = __ffma2_rn(zp[i], zp[i], dist2[i]);
       }
-      if constexpr (PW) qs2 = __fadd2_rn(qs2, q);
     };
     constexpr bool kPackedB = (G == 2);
     if constexpr (kPackedB) {
@@ -495,9 +513,13 @@ __global__ void __launch_bounds__(all_threads(N), all_ctas_per_sm(N)) rows_all_k
     for (int i = 0; i < N; ++i) {
       float dv = dist[i];
       if constexpr (kPackedB) dv += dist2[i].x + dist2[i].y;
-      if constexpr (PW && !KL) {   // sum_{j != i} (z_i - z_j)^2 = n z'_i^2 + sum_j z'_j^2
-        float qv = qs;
-        if constexpr (kPackedB) qv += qs2.x + qs2.y;
+      if constexpr (PW && !KL) {   // sum_{j != i} (z_i - z_j)^2 = n z'_i^2 + sum_j z'_j^2, the second sum from all models' z'^2
+        float qv = 0.f;
+#pragma unroll
+        for (int j = 0; j < N; ++j) {
+          qv += dist[j];
+          if constexpr (kPackedB) qv += dist2[j].x + dist2[j].y;
+        }
         dv = fmaf((float)N, dv, qv);
       }
       const float dw = warp_sum(dv);
