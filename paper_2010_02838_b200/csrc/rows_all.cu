@@ -119,24 +119,18 @@ __global__ void __launch_bounds__(all_threads(N), all_ctas_per_sm(N)) rows_all_k
   const bool t_one = a.temperature == 1.f;
   const float ckl = with_term ? w * a.alpha * a.temperature / (float)(N - 1) : 0.f;  // (n t_i - Q) -> w alpha dD_i/dz_i
 
-  if (tid == 0) sh.next_row[0] = (long long)atomicAdd(&a.hdr->next_row, 1u);
+  stream_draw_row(&sh.next_row[0], a.hdr, 0, tid);
   __syncthreads();
   int v = 0;  // valid rows done by this CTA
   for (int it = 0;; ++it) {
     const long long r = sh.next_row[it & 1];
     if (r >= R) break;
-    if (tid == 0) sh.next_row[(it + 1) & 1] = (long long)atomicAdd(&a.hdr->next_row, 1u);
-    const RowGeom g = row_geom<T>(r, a.row_stride, C);
-    const int64_t row_off = r * a.row_stride;  // in elements
-    const int n_int = g.seg_hi > g.seg_lo ? g.seg_hi - g.seg_lo : 0;    // segments wholly inside the row
-    const int cnt = n_int > tid ? (n_int - tid + NT - 1) / NT : 0;     // of which this thread has cnt: seg_lo + tid + NT * i
-    const int s0 = g.seg_lo + tid;
-    const bool edge_head = (tid == 0) && g.seg_lo > 0;
-    const bool edge_tail = (tid == 32) && g.seg_hi < g.n_seg && (g.n_seg > 1 || g.seg_lo == 0);
-    const bool edge = edge_head || edge_tail;
-    const int edge_seg = edge_head ? 0 : g.n_seg - 1;
-    const int y = a.labels[r];
-    const bool valid = (a.mask == nullptr || a.mask[r] != 0) && y >= 0 && (int64_t)y < C;
+    stream_draw_row(&sh.next_row[(it + 1) & 1], a.hdr, 0, tid);
+    const StreamRow row = stream_row<T, NT>(r, r, a.row_stride, C, a.labels, a.mask, tid);
+    const RowGeom g = row.g;
+    const int64_t row_off = row.row_off;  // in elements
+    const int cnt = row.cnt, s0 = row.s0, y = row.y, edge_seg = row.edge_seg;
+    const bool edge = row.edge;
     const T* z_row[N];
     const uint4* z_img[N];
 #pragma unroll
@@ -146,21 +140,10 @@ __global__ void __launch_bounds__(all_threads(N), all_ctas_per_sm(N)) rows_all_k
     }
     const bool want_grad = a.grad[0] != nullptr;
 
-    if (!valid) {  // masked row: zero gradient rows, no loss, no counts; nothing is read
+    if (!row.valid) {  // masked row: zero gradient rows, no loss, no counts; nothing is read
       if (want_grad) {
 #pragma unroll
-        for (int i = 0; i < N; ++i) {
-          T* g_row = reinterpret_cast<T*>(a.grad[i]) + row_off;
-          uint4* g_img = reinterpret_cast<uint4*>(g_row - g.head);
-          for (int k = 0; k < cnt; ++k) g_img[s0 + k * NT] = make_uint4(0u, 0u, 0u, 0u);
-          if (edge) {
-#pragma unroll
-            for (int e = 0; e < V; ++e) {
-              const int64_t c = (int64_t)edge_seg * V - g.head + e;
-              if (c >= 0 && c < C) g_row[c] = Elem<T>::from_f32(0.f);
-            }
-          }
-        }
+        for (int i = 0; i < N; ++i) stream_zero_row<T, NT>(reinterpret_cast<T*>(a.grad[i]) + row_off, row, C);
       }
       if (tid < N) { a.row_loss[(int64_t)tid * R + r] = 0.f; a.row_flags[(int64_t)tid * R + r] = 0u; }
       __syncthreads();  // orders the row-id hand-over
@@ -548,13 +531,8 @@ __global__ void __launch_bounds__(all_threads(N), all_ctas_per_sm(N)) rows_all_k
     ++v;
   }
 
-  // ---------------- all rows of this CTA are written: scheduler reset
-  __threadfence();
-  __syncthreads();
-  if (tid == 0) {
-    const unsigned int prev = atomicAdd(&a.hdr->sched_done, 1u);
-    if (prev == gridDim.x - 1) { a.hdr->next_row = 0u; a.hdr->sched_done = 0u; __threadfence(); }  // ready for the next launch
-  }
+  // ---------------- all rows of this CTA are written: scheduler reset (the final reduction is a kernel of its own)
+  stream_last_cta(a.hdr, &sh.last_flag, tid);
 }
 
 // Final reduction of the n models: block i sums model i's row losses and counts its flag bits.

@@ -28,7 +28,6 @@ __global__ void __launch_bounds__(stream_threads(P), stream_ctas_per_sm(P)) rows
   constexpr int V = SegOps<T>::V;
   constexpr int H = SegOps<T>::H;
   constexpr int PD = P > 0 ? P : 1;
-  constexpr int ES = (int)sizeof(T);
   constexpr int NT = stream_threads(P);
   constexpr int kAhead = stream_ahead(P);
   constexpr int kStreamWarps = NT / 32;
@@ -52,41 +51,25 @@ __global__ void __launch_bounds__(stream_threads(P), stream_ctas_per_sm(P)) rows
   const float2 l2e2 = make_float2(kLog2e, kLog2e);
   const float2 neg1 = make_float2(-1.f, -1.f);
 
-  if (tid == 0) sh.next_row[0] = a.row_begin + (long long)atomicAdd(&a.hdr->next_row, 1u);
+  stream_draw_row(&sh.next_row[0], a.hdr, a.row_begin, tid);
   __syncthreads();
   int v = 0;  // valid rows done by this CTA
   for (int it = 0;; ++it) {
     const long long r = sh.next_row[it & 1];
     if (r >= a.row_end) break;
-    if (tid == 0) sh.next_row[(it + 1) & 1] = a.row_begin + (long long)atomicAdd(&a.hdr->next_row, 1u);
-    const int64_t lr = r - a.row_begin;
-    const RowGeom g = row_geom<T>(lr, a.row_stride, C);
-    const int64_t row_off = lr * a.row_stride;  // in elements
+    stream_draw_row(&sh.next_row[(it + 1) & 1], a.hdr, a.row_begin, tid);
+    const StreamRow row = stream_row<T, NT>(r - a.row_begin, r, a.row_stride, C, a.labels, a.mask, tid);
+    const RowGeom g = row.g;
+    const int64_t row_off = row.row_off;  // in elements
     const T* __restrict__ z_row = reinterpret_cast<const T*>(a.own) + row_off;
     T* __restrict__ g_row = a.grad ? reinterpret_cast<T*>(a.grad) + row_off : nullptr;
     const uint4* __restrict__ z_img = reinterpret_cast<const uint4*>(z_row - g.head);
     uint4* __restrict__ g_img = g_row ? reinterpret_cast<uint4*>(g_row - g.head) : nullptr;
-    const int n_int = g.seg_hi > g.seg_lo ? g.seg_hi - g.seg_lo : 0;    // segments wholly inside the row
-    const int cnt = n_int > tid ? (n_int - tid + NT - 1) / NT : 0;     // of which this thread has cnt: seg_lo + tid + NT * i
-    const int s0 = g.seg_lo + tid;
-    // ragged segments: thread 0 takes the first, thread 32 the last
-    const bool edge_head = (tid == 0) && g.seg_lo > 0;
-    const bool edge_tail = (tid == 32 % NT) && g.seg_hi < g.n_seg && (g.n_seg > 1 || g.seg_lo == 0);
-    const int y = a.labels[r];
-    const bool valid = (a.mask == nullptr || a.mask[r] != 0) && y >= 0 && (int64_t)y < C;
+    const int cnt = row.cnt, s0 = row.s0, y = row.y;
+    const bool edge_head = row.edge_head, edge_tail = row.edge_tail;
 
-    if (!valid) {  // masked row: zero gradient, no loss, no counts; nothing is read
-      if (g_img) {
-        for (int i = 0; i < cnt; ++i) g_img[s0 + i * NT] = make_uint4(0u, 0u, 0u, 0u);
-        if (edge_head || edge_tail) {
-          const int s = edge_head ? 0 : g.n_seg - 1;
-#pragma unroll
-          for (int i = 0; i < V; ++i) {
-            const int64_t c = (int64_t)s * V - g.head + i;
-            if (c >= 0 && c < C) g_row[c] = Elem<T>::from_f32(0.f);
-          }
-        }
-      }
+    if (!row.valid) {  // masked row: zero gradient, no loss, no counts; nothing is read
+      if (g_row) stream_zero_row<T, NT>(g_row, row, C);
       if (tid == 0) { a.row_loss[r] = 0.f; a.row_flags[r] = 0u; }
       __syncthreads();  // orders the row-id hand-over
       continue;
@@ -459,15 +442,7 @@ __global__ void __launch_bounds__(stream_threads(P), stream_ctas_per_sm(P)) rows
   }
 
   // ---------------- all rows of this CTA are written: scheduler reset and final reduction
-  __threadfence();
-  __syncthreads();
-  if (tid == 0) {
-    const unsigned int prev = atomicAdd(&a.hdr->sched_done, 1u);
-    sh.last_flag = (prev == gridDim.x - 1);
-    if (sh.last_flag) { a.hdr->next_row = 0u; a.hdr->sched_done = 0u; __threadfence(); }  // ready for the next launch
-  }
-  __syncthreads();
-  if (a.fused_finalize && sh.last_flag) {
+  if (stream_last_cta(a.hdr, &sh.last_flag, tid) && a.fused_finalize) {
     __threadfence();
     finalize_cta(a, sh.fin);
   }

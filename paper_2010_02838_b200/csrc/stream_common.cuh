@@ -56,6 +56,75 @@ __device__ __forceinline__ uint64_t make_policy_stream() {
   return pol;
 }
 
+// ------------------------------------------------------------------ the persistent-row skeleton
+// The direct-load kernels run a fixed number of CTAs that draw row ids from a counter in the workspace
+// header.  These pieces are the same in all of them.
+
+// How one CTA of NT threads sees one row: geometry of the row image, this thread's share of the whole
+// segments (s0, s0 + NT, ...: cnt of them), which thread does a ragged first / last segment element by
+// element (thread 0 / thread 32), the label and whether the row takes part.
+struct StreamRow {
+  RowGeom g;
+  int64_t row_off;   // first element of the row relative to the tensor (local row * pitch)
+  int cnt, s0;
+  bool edge_head, edge_tail, edge;
+  int edge_seg;
+  int y;
+  bool valid;
+};
+template <typename T, int NT>
+__device__ __forceinline__ StreamRow stream_row(int64_t local_row, long long global_row, int64_t row_stride, int64_t C,
+                                                const int32_t* labels, const uint8_t* mask, int tid) {
+  StreamRow w;
+  w.g = row_geom<T>(local_row, row_stride, C);
+  w.row_off = local_row * row_stride;
+  const int n_int = w.g.seg_hi > w.g.seg_lo ? w.g.seg_hi - w.g.seg_lo : 0;   // segments wholly inside the row
+  w.cnt = n_int > tid ? (n_int - tid + NT - 1) / NT : 0;
+  w.s0 = w.g.seg_lo + tid;
+  w.edge_head = (tid == 0) && w.g.seg_lo > 0;
+  w.edge_tail = (tid == 32) && w.g.seg_hi < w.g.n_seg && (w.g.n_seg > 1 || w.g.seg_lo == 0);
+  w.edge = w.edge_head || w.edge_tail;
+  w.edge_seg = w.edge_head ? 0 : w.g.n_seg - 1;
+  w.y = labels[global_row];
+  w.valid = (mask == nullptr || mask[global_row] != 0) && w.y >= 0 && (int64_t)w.y < C;
+  return w;
+}
+
+// The all-zero gradient row of a masked row: whole segments by 16-byte stores, ragged ones element by element.
+template <typename T, int NT>
+__device__ __forceinline__ void stream_zero_row(T* __restrict__ g_row, const StreamRow& w, int64_t C) {
+  constexpr int V = SegOps<T>::V;
+  uint4* g_img = reinterpret_cast<uint4*>(g_row - w.g.head);
+  for (int i = 0; i < w.cnt; ++i) g_img[w.s0 + i * NT] = make_uint4(0u, 0u, 0u, 0u);
+  if (w.edge) {
+#pragma unroll
+    for (int i = 0; i < V; ++i) {
+      const int64_t c = (int64_t)w.edge_seg * V - w.g.head + i;
+      if (c >= 0 && c < C) g_row[c] = Elem<T>::from_f32(0.f);
+    }
+  }
+}
+
+// Row ids: thread 0 draws the next id while the CTA works on the current one; two slots in shared memory
+// alternate, and every row passes at least one __syncthreads() between the write and the reads of a slot.
+__device__ __forceinline__ void stream_draw_row(long long* slot, WsHeader* hdr, long long row_begin, int tid) {
+  if (tid == 0) *slot = row_begin + (long long)atomicAdd(&hdr->next_row, 1u);
+}
+
+// Called by every thread once the CTA's rows are written.  Returns true in the CTA that arrives last; that CTA has
+// put the row counter back to zero for the next launch.  `flag` is one int of shared memory.
+__device__ __forceinline__ bool stream_last_cta(WsHeader* hdr, int* flag, int tid) {
+  __threadfence();
+  __syncthreads();
+  if (tid == 0) {
+    const unsigned int prev = atomicAdd(&hdr->sched_done, 1u);
+    *flag = (prev == gridDim.x - 1);
+    if (*flag) { hdr->next_row = 0u; hdr->sched_done = 0u; __threadfence(); }
+  }
+  __syncthreads();
+  return *flag != 0;
+}
+
 // First column of segment `s` of the row image whose value equals m, or INT_MAX; reads single elements.
 template <typename T>
 __device__ __noinline__ int first_equal_global(const T* __restrict__ z_row, int s, int head, int64_t C, float m) {
