@@ -30,7 +30,10 @@ namespace codistill {
 
 constexpr int kAllMax = CODISTILL_ALL_MAX_MODELS;
 __host__ __device__ constexpr int all_threads(int n) { return n >= 5 ? 128 : 256; }
-__host__ __device__ constexpr int all_ctas_per_sm(int n) { return n >= 5 ? 4 : 3; }
+// CTAs per SM.  Five and more models run 128-thread CTAs: four per SM for the KL form, three for the MSE forms (168
+// registers per thread and next to no spills instead of 128 with spills: workload 5, all 8 models, 6.94 -> 6.45 ms;
+// the KL form was 10 % slower that way, and two CTAs per SM were slower for both).
+__host__ __device__ constexpr int all_ctas_per_sm(int n, bool kl) { return n >= 5 ? (kl ? 4 : 3) : 3; }
 
 struct AllArgs {
   const void* model[kAllMax];
@@ -90,7 +93,7 @@ __device__ __forceinline__ float exp_nat(float x) {
 }
 
 template <typename T, int N, bool PW, bool KL>
-__global__ void __launch_bounds__(all_threads(N), all_ctas_per_sm(N)) rows_all_kernel(const __grid_constant__ AllArgs a) {
+__global__ void __launch_bounds__(all_threads(N), all_ctas_per_sm(N, KL)) rows_all_kernel(const __grid_constant__ AllArgs a) {
   constexpr int V = SegOps<T>::V;
   constexpr int G = WordOps<T>::G;
   constexpr int NT = all_threads(N);
@@ -570,7 +573,7 @@ static AllLayout all_layout(int n, int64_t rows) {
 
 template <typename T, int N>
 static cudaError_t all_launch_n(const AllArgs& a, int num_sms, cudaStream_t stream) {
-  const int64_t slots = (int64_t)num_sms * all_ctas_per_sm(N);
+  const int64_t slots = (int64_t)num_sms * all_ctas_per_sm(N, a.temperature > 0.f);
   const int grid = (int)(a.rows < slots ? a.rows : slots);
   cudaError_t e;
   if (a.temperature > 0.f)  // KL distance, pairwise over the peers
